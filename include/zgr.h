@@ -1,0 +1,138 @@
+/*
+ * zgr.h - C ABI of the ZGR hot path: the zeroth-order (ZOO) step with cloud-guided gradient
+ * rectification of CooperLLM, as hand-written CUDA for NVIDIA B200 (sm_100a).
+ *
+ * What one step does (Sec. 3.2, Eq. (perturbation), Eq. (grad), Algorithm 1).  For every weight
+ * tensor theta_l (rows x cols, row-major) the hybrid perturbation
+ *
+ *      z_l = a * Z_l  +  b * U_l * G_l
+ *
+ * is regenerated on the fly from a 64-bit seed: Z_l is isotropic Gaussian noise, U_l (rows x r,
+ * orthonormal columns) is the cloud-supplied gradient subspace of that tensor and G_l (r x cols)
+ * holds the guided coefficients, either drawn from the seed or delivered compressed (Sec. 3.4,
+ * DTC).  A step is three in-place sweeps over the weights and never stores z:
+ *
+ *      zgr_perturb(seed, +eps)            theta <- rnd(theta + eps z)       forward pass -> L+
+ *      zgr_perturb(seed, -2 eps)          theta <- rnd(theta - 2 eps z)     forward pass -> L-
+ *      zgr_restore_update(seed, L+, L-, lr)
+ *                                         theta <- rnd(theta + (eps - lr (L+ - L-)/(2 eps)) z)
+ *
+ * Conventions.
+ *   - Every `void* stream` is a cudaStream_t (NULL = the legacy default stream).  Sweeps are
+ *     enqueued on it and return without synchronising.
+ *   - "device" pointers are CUDA device addresses on the current device; the library never
+ *     dereferences them on the host and never frees them.  They are borrowed for the life of the
+ *     context.
+ *   - All functions return 0 on success or a negative ZGR_E* code.  Arguments are validated before
+ *     anything is launched: a call that fails validation leaves the weights untouched.
+ *   - A context is bound to the device that is current when zgr_init is called and is not
+ *     thread-safe; use one per thread or serialise calls.
+ */
+#ifndef ZGR_H_
+#define ZGR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ZGR_MAX_RANK 64 /* largest subspace rank r per tensor */
+
+enum { ZGR_OK = 0, ZGR_EINVAL = -1, ZGR_ESTATE = -2, ZGR_ECUDA = -3, ZGR_ENOMEM = -4 };
+
+/* storage type of a weight tensor; arithmetic is fp32, one round-to-nearest-even per sweep */
+enum { ZGR_F32 = 0, ZGR_F16 = 1, ZGR_BF16 = 2 };
+
+/* Normalisation of Eq. (perturbation), with n := d = total parameters and m := K = total guided
+ * coefficients (sum of rank * cols over tensors that have a subspace):
+ *   ZGR_SCALE_PAPER  a = sqrt(alpha/d),  b = sqrt((1-alpha)/K)          (E|z|^2 = 1)
+ *   ZGR_SCALE_UNIT   a = sqrt(alpha),    b = sqrt((1-alpha) d/K)        (E|z|^2 = d; alpha = 1 is
+ *                                                                       exactly the z of Eq. (ZOO)) */
+enum { ZGR_SCALE_PAPER = 0, ZGR_SCALE_UNIT = 1 };
+
+/* Stream tags of the counter-based generator (fourth counter word). */
+enum { ZGR_TAG_ISO = 0, ZGR_TAG_COEFF = 1 };
+
+typedef struct zgr_ctx zgr_ctx; /* opaque; created by zgr_init, released by zgr_destroy */
+
+/* One weight tensor.  1-D tensors are given as rows = 1, cols = length, U = NULL, rank = 0. */
+typedef struct {
+  void* data;       /* device; rows*cols elements of `dtype`, row-major, contiguous, updated in place.
+                       Must be aligned to the element size; 16-byte alignment and cols a multiple of
+                       16 bytes' worth of elements select the vectorised kernels */
+  int64_t rows;     /* m_l >= 1 */
+  int64_t cols;     /* n_l >= 1 */
+  int32_t dtype;    /* ZGR_F32 | ZGR_F16 | ZGR_BF16 */
+  int32_t rank;     /* r_l in [0, ZGR_MAX_RANK]; 0 = isotropic noise only */
+  const float* U;   /* device; rows x rank fp32 row-major, orthonormal columns (not checked, not
+                       re-orthonormalised); NULL iff rank == 0 */
+} zgr_tensor;
+
+typedef struct {
+  double alpha;            /* mixing ratio of Eq. (perturbation), in [0, 1] */
+  double eps;              /* perturbation scale epsilon > 0 of Eq. (ZOO) */
+  int32_t scale_mode;      /* ZGR_SCALE_PAPER | ZGR_SCALE_UNIT */
+  int32_t bits_per_normal; /* 32: one generator block per 4 elements; 16: one per 8 elements */
+} zgr_config;
+
+/* Build a context over `n` tensors (Algorithm 1, "Require": model, epsilon, alpha, subspace).
+ * `tensors` and `cfg` are host pointers, copied.  Tensor l gets generator tensor-id l.
+ * Allocates only the library's own descriptor and work tables on the current device.
+ * ZGR_EINVAL: null argument, n <= 0, bad dtype/rank/shape, misaligned data, alpha outside [0,1],
+ * eps <= 0 or not finite, unknown scale_mode or bits_per_normal.  ZGR_ECUDA / ZGR_ENOMEM: no usable
+ * device or allocation failure (also the answer on a machine without a GPU). */
+int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_config* cfg);
+
+/* theta_l <- rnd(theta_l + scale * z_l(seed)) for every tensor (Algorithm 1, "Compute loss
+ * difference": W + eps z_h, then W - eps z_h, reached by scale = +eps followed by scale = -2 eps).
+ * The context remembers `seed` and the sum of the scales applied under it.
+ * ZGR_EINVAL: scale not finite.  ZGR_ESTATE: a different seed is still active (its
+ * restore_update has not been called). */
+int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream);
+
+/* Undo the net perturbation of `seed` and take the projected-gradient step in the same sweep
+ * (Eq. (grad); Algorithm 1 "Recover gradient", "Update"):
+ *     g = (loss_plus - loss_minus) / (2 eps),   theta_l <- rnd(theta_l + (-net - lr g) z_l(seed)).
+ * lr = 0 is a pure restore.  Scalars are combined in double on the host and passed to the kernel
+ * as fp32.  ZGR_EINVAL: a loss or lr is not finite.  ZGR_ESTATE: `seed` is not the active seed. */
+int zgr_restore_update(zgr_ctx* ctx, uint64_t seed, double loss_plus, double loss_minus, double lr, void* stream);
+
+/* Deliver the guided coefficients of one tensor compressed (Sec. 3.4, DTC): from now on
+ *     G_l[k][c] = scale[k] * (q[k][c] - zero[k])       (x = lambda (x_quant - delta))
+ * replaces the seed-drawn G_l.  q: device, rank x cols int8 row-major; scale: device, rank fp32;
+ * zero: device, rank fp32, or NULL for delta = 0; bits must be 8.  Pointers are borrowed, not copied.
+ * ZGR_EINVAL: bad tensor index, tensor without subspace, null q/scale, bits != 8.
+ * ZGR_ESTATE: a perturbation is active (the coefficients must not change between a perturb and
+ * its restore_update). */
+int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits);
+
+/* Back to seed-drawn coefficients for `tensor` (Algorithm 1, "Sample z_g").  Errors as above. */
+int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor);
+
+/* Norm bookkeeping for the adaptive choice of alpha mentioned in Sec. 1: for each tensor l,
+ * out[3l+0] = sum (a Z_l)^2, out[3l+1] = sum (b U_l G_l)^2, out[3l+2] = sum z_l^2 for `seed`.
+ * Reads no weights.  `out` is a HOST array of 3*n doubles; the call synchronises `stream`. */
+int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream);
+
+/* Test hooks.  zgr_debug_philox writes n_blocks raw generator blocks (4 uint32 each) of stream
+ * (seed, tensor, tag) starting at first_block to dev_out (device).  zgr_debug_z writes z_l(seed) as
+ * fp32 (rows*cols, device) using the same kernels as the sweeps (it sweeps a zeroed fp32 scratch
+ * image of the tensor with scale 1). */
+int zgr_debug_philox(zgr_ctx* ctx, uint64_t seed, int32_t tensor, int32_t tag, uint64_t first_block, int64_t n_blocks,
+                     uint32_t* dev_out, void* stream);
+int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, void* stream);
+
+/* Introspection: mixing scalars a, b in double; active seed / net scale (active = 0 when idle);
+ * number of kernel launches issued by this context so far. */
+int zgr_get_scalars(const zgr_ctx* ctx, double* a, double* b);
+int zgr_get_state(const zgr_ctx* ctx, int32_t* active, uint64_t* seed, double* net_scale);
+int64_t zgr_launch_count(const zgr_ctx* ctx);
+
+void zgr_destroy(zgr_ctx* ctx);
+const char* zgr_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZGR_H_ */
