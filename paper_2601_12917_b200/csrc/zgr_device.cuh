@@ -1,0 +1,234 @@
+// Device-side building blocks of the ZGR sweeps: the counter-based generator, the Gaussian
+// transform, and 8-element ("octet") access to the three storage types.
+#ifndef ZGR_DEVICE_CUH_
+#define ZGR_DEVICE_CUH_
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include "zgr_internal.h"
+
+namespace zgr {
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11).  The paper asks only that client and edge server
+// regenerate the same perturbation from a shared seed (Algorithm 1); a counter-based generator
+// makes every element a pure function of (seed, tensor, stream tag, element index), so any tiling
+// of the sweep produces the same bits.  Round keys arrive precomputed in the kernel parameters and
+// become constant-bank operands of the xors.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys& k,
+                                              uint32_t (&x)[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = static_cast<uint64_t>(0xD2511F53u) * c0;
+    const uint64_t p1 = static_cast<uint64_t>(0xCD9E8D57u) * c2;
+    const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ k.k0[r];
+    const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ k.k1[r];
+    c1 = static_cast<uint32_t>(p1);
+    c3 = static_cast<uint32_t>(p0);
+    c0 = n0;
+    c2 = n2;
+  }
+  x[0] = c0; x[1] = c1; x[2] = c2; x[3] = c3;
+}
+
+__device__ __forceinline__ void philox_block(uint64_t j, uint32_t tensor, uint32_t tag, const PhiloxKeys& k, uint32_t (&x)[4]) {
+  philox4x32_10(static_cast<uint32_t>(j), static_cast<uint32_t>(j >> 32), tensor, tag, k, x);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Box-Muller on odd-numerator uniforms  u = (2k+1) / 2^(nb+1),  k an nb-bit field (nb = 23 or 16):
+//     n0 = s rho cos(phi),  n1 = s rho sin(phi),   rho = sqrt(-2 ln u1),  phi = 2 pi u2,
+// with the output scale s folded in: |s| goes under the square root, the sign of s becomes a half
+// turn of the angle.  The field k is OR-ed into the mantissa of 1.0f, so t = 1 + k 2^-23 costs no
+// conversion instruction, and u1 = t + (2^-(nb+1) - 1) is exact in fp32.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float lg2_approx(float x) {
+  float r;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float r;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float sin_approx(float x) {
+  float r;
+  asm("sin.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float cos_approx(float x) {
+  float r;
+  asm("cos.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+
+// m1, m2: the two uniform fields already placed in mantissa position (bits 0..22).
+// PRECISE selects a radius that stays accurate where u1 is close to 1: the hardware log2 has an
+// absolute error of about 2^-22 there, which the square root would amplify for the smallest radii;
+// for 1 - u1 < 2^-6 the series -2 ln(1-v) = 2v + v^2 + (2/3) v^3 is used instead.  fp32 weights
+// need it for their 1e-6 tolerance; 16-bit weights do not.
+template <bool PRECISE>
+__device__ __forceinline__ void box_muller(uint32_t m1, uint32_t m2, const NormalScale& ns, float& n0, float& n1) {
+  const float u1 = __uint_as_float(0x3F800000u | m1) + ns.u1_off;
+  const float t2 = __uint_as_float(0x3F800000u | m2);
+  float r2 = fabsf(ns.kr * lg2_approx(u1));
+  if (PRECISE) {
+    const float v = 1.0f - u1;
+    const float series = v * fmaf(v, fmaf(v, 0.66666667f, 1.0f), 2.0f) * ns.s2;
+    r2 = v < 0.015625f ? series : r2;
+  }
+  const float rho = sqrt_approx(r2);
+  const float phi = fmaf(t2, 6.28318530717958647692f, ns.phase);
+  n0 = rho * cos_approx(phi);
+  n1 = rho * sin_approx(phi);
+}
+
+// Eight consecutive normals of stream (tensor, tag) starting at element e (a multiple of 8), each
+// already multiplied by the scale folded into `ns`.
+//   BITS == 32: blocks e/4 and e/4+1; words (x0,x1) -> normals 0,1 and (x2,x3) -> normals 2,3.
+//   BITS == 16: block e/8; word w -> normals 2w, 2w+1 from its high and low 16 bits.
+template <int BITS, bool PRECISE>
+__device__ __forceinline__ void normals8(const PhiloxKeys& keys, uint32_t tensor, uint32_t tag, uint64_t e, const NormalScale& ns,
+                                         float (&z)[8]) {
+  uint32_t x[4];
+  if (BITS == 32) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      philox_block((e >> 2) + h, tensor, tag, keys, x);
+      box_muller<PRECISE>(x[0] >> 9, x[1] >> 9, ns, z[4 * h + 0], z[4 * h + 1]);
+      box_muller<PRECISE>(x[2] >> 9, x[3] >> 9, ns, z[4 * h + 2], z[4 * h + 3]);
+    }
+  } else {
+    philox_block(e >> 3, tensor, tag, keys, x);
+#pragma unroll
+    for (int w = 0; w < 4; ++w)
+      box_muller<PRECISE>((x[w] >> 9) & 0x7FFF80u, (x[w] << 7) & 0x7FFF80u, ns, z[2 * w], z[2 * w + 1]);
+  }
+}
+
+// One normal at an arbitrary element index (ragged tails and the unaligned fallback kernels).
+template <int BITS, bool PRECISE>
+__device__ __forceinline__ float normal1(const PhiloxKeys& keys, uint32_t tensor, uint32_t tag, uint64_t e, const NormalScale& ns) {
+  uint32_t x[4];
+  float n0, n1;
+  if (BITS == 32) {
+    philox_block(e >> 2, tensor, tag, keys, x);
+    const int pair = static_cast<int>(e & 3) >> 1;
+    box_muller<PRECISE>((pair ? x[2] : x[0]) >> 9, (pair ? x[3] : x[1]) >> 9, ns, n0, n1);
+  } else {
+    philox_block(e >> 3, tensor, tag, keys, x);
+    const int w = static_cast<int>(e & 7) >> 1;
+    const uint32_t word = w == 0 ? x[0] : (w == 1 ? x[1] : (w == 2 ? x[2] : x[3]));
+    box_muller<PRECISE>((word >> 9) & 0x7FFF80u, (word << 7) & 0x7FFF80u, ns, n0, n1);
+  }
+  return (e & 1) ? n1 : n0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Storage access: eight contiguous elements as fp32, 128-bit transactions, streaming cache hints
+// (every weight is touched exactly once per sweep).  Stores round to nearest even.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+struct Storage;
+
+template <>
+struct Storage<float> {
+  static __device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+    const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+  static __device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(v[0], v[1], v[2], v[3]));
+    __stcs(reinterpret_cast<float4*>(p) + 1, make_float4(v[4], v[5], v[6], v[7]));
+  }
+  static __device__ __forceinline__ float load1(const float* p) { return *p; }
+  static __device__ __forceinline__ void store1(float* p, float v) { *p = v; }
+};
+
+template <>
+struct Storage<__half> {
+  static __device__ __forceinline__ void load8(const __half* p, float (&v)[8]) {
+    const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+      v[2 * i] = f.x;
+      v[2 * i + 1] = f.y;
+    }
+  }
+  static __device__ __forceinline__ void store8(__half* p, const float (&v)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __half2 h = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+  }
+  static __device__ __forceinline__ float load1(const __half* p) { return __half2float(*p); }
+  static __device__ __forceinline__ void store1(__half* p, float v) { *p = __float2half_rn(v); }
+};
+
+template <>
+struct Storage<__nv_bfloat16> {
+  static __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+    const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+  static __device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+  }
+  static __device__ __forceinline__ float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+  static __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Guided coefficients G_l[k][c .. c+7], multiplied by `cb`  (Algorithm 1 "Sample z_g"; Sec. 3.4 for
+// the compressed form  x = lambda (x_quant - delta)).
+// ---------------------------------------------------------------------------------------------
+template <int BITS, bool PRECISE>
+__device__ __forceinline__ void coeffs8(const TensorDesc& td, const PhiloxKeys& keys, const NormalScale& unit, float cb, int k,
+                                        int64_t c, float (&g)[8]) {
+  if (td.q != nullptr) {
+    const float lambda = td.qscale[k] * cb;
+    const float delta = td.qzero ? td.qzero[k] : 0.0f;
+    const int8_t* src = td.q + static_cast<int64_t>(k) * td.cols + c;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) g[i] = lambda * (static_cast<float>(src[i]) - delta);
+  } else {
+    normals8<BITS, PRECISE>(keys, static_cast<uint32_t>(td.id), 1u, static_cast<uint64_t>(k) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(c),
+                            unit, g);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) g[i] *= cb;
+  }
+}
+
+template <int BITS, bool PRECISE>
+__device__ __forceinline__ float coeff1(const TensorDesc& td, const PhiloxKeys& keys, const NormalScale& unit, float cb, int k, int64_t c) {
+  if (td.q != nullptr) {
+    const float delta = td.qzero ? td.qzero[k] : 0.0f;
+    return td.qscale[k] * cb * (static_cast<float>(td.q[static_cast<int64_t>(k) * td.cols + c]) - delta);
+  }
+  return cb * normal1<BITS, PRECISE>(keys, static_cast<uint32_t>(td.id), 1u,
+                                     static_cast<uint64_t>(k) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(c), unit);
+}
+
+}  // namespace zgr
+#endif  // ZGR_DEVICE_CUH_

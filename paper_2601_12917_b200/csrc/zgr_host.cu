@@ -1,0 +1,477 @@
+// Host side of the ZGR library: context, validation, work planning and the C entry points
+// declared in include/zgr.h.  Everything numerical happens in the kernels; the host only
+// combines the step scalars in double (Eq. (grad), Eq. (perturbation)) and hands them over as fp32.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <map>
+#include <new>
+#include <vector>
+
+#include "zgr.h"
+#include "zgr_internal.h"
+#include "zgr_kernels.h"
+
+using namespace zgr;
+
+namespace {
+
+struct Group {
+  KernelChoice kc;
+  std::vector<WorkItem> items;
+  WorkItem* d_items = nullptr;
+  int grid = 0;
+};
+
+int dtype_bytes(int dt) { return dt == ZGR_F32 ? 4 : 2; }
+
+}  // namespace
+
+struct zgr_ctx {
+  int device = 0;
+  int sm_count = 0;
+  zgr_config cfg{};
+  double a = 0, b = 0;
+  int64_t d = 0, K = 0;
+  std::vector<TensorDesc> descs;      // host mirror of the device table
+  TensorDesc* d_descs = nullptr;
+  bool descs_dirty = false;
+  std::vector<void*> owned;           // device allocations made by the library
+  std::vector<Group> groups;          // sweep plan
+  std::vector<WorkItem> stats_items;  // plan of the norm kernel
+  WorkItem* d_stats_items = nullptr;
+  double* d_stats = nullptr;
+  bool active = false;
+  uint64_t seed = 0;
+  double net = 0;
+  int sticky = 0;                     // first CUDA failure, returned by every later call
+  int64_t launches = 0;
+};
+
+namespace {
+
+PhiloxKeys make_keys(uint64_t seed) {
+  PhiloxKeys k;
+  uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    k.k0[r] = k0;
+    k.k1[r] = k1;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return k;
+}
+
+NormalScale make_scale(double s, int bits) {
+  const double kTwoPi = 6.283185307179586476925286766559;
+  const int nb = bits == 32 ? 23 : 16;
+  const double off = std::ldexp(1.0, -(nb + 1)) - 1.0;
+  NormalScale ns;
+  ns.kr = static_cast<float>(-2.0 * std::log(2.0) * s * s);
+  ns.s2 = static_cast<float>(s * s);
+  ns.phase = static_cast<float>(kTwoPi * off + (s >= 0 ? -kTwoPi : -0.5 * kTwoPi));
+  ns.u1_off = static_cast<float>(off);
+  return ns;
+}
+
+int blocks_per_sm(int path) {
+  switch (path) {
+    case PATH_ISO: return 6;
+    case PATH_GENERIC: return 4;
+    default: return 2;
+  }
+}
+
+// Split the tensors listed in `which` into work items, grouped by the kernel that serves them.
+void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, bool guided_on, int bits, int sm_count,
+          std::vector<Group>& out) {
+  int64_t total = 0;
+  for (int l : which) total += descs[l].rows * descs[l].cols;
+  // elements per item: enough items for ~16 rounds over the resident CTAs, but large enough that the
+  // coefficient strip of an item is a small fraction of its work
+  int64_t target = total / (static_cast<int64_t>(sm_count) * 2 * 16);
+  target = std::min<int64_t>(std::max<int64_t>(target, 16384), 524288);
+
+  std::map<std::tuple<int, int, int>, size_t> index;  // (path, dtype, kpad) -> group
+  auto group_for = [&](int path, int dtype, int kpad) -> Group& {
+    auto key = std::make_tuple(path, dtype, kpad);
+    auto it = index.find(key);
+    if (it == index.end()) {
+      index[key] = out.size();
+      Group g;
+      g.kc = KernelChoice{path, dtype, kpad, bits};
+      out.push_back(std::move(g));
+      return out.back();
+    }
+    return out[it->second];
+  };
+
+  for (int l : which) {
+    const TensorDesc& t = descs[l];
+    const int eb = dtype_bytes(t.dtype);
+    const bool aligned = (reinterpret_cast<uintptr_t>(t.data) & 15) == 0;
+    const bool guided = guided_on && t.rank > 0;
+    if (!guided) {
+      Group& g = group_for(PATH_ISO, t.dtype, 0);
+      const int64_t n = t.rows * t.cols;
+      const int64_t chunk = std::max<int64_t>(8, (target / 8) * 8);
+      for (int64_t e0 = 0; e0 < n; e0 += chunk)
+        g.items.push_back(WorkItem{l, aligned ? 1 : 0, e0, std::min(chunk, n - e0), 0});
+      continue;
+    }
+    const bool vec = aligned && (t.cols % 8 == 0);
+    int path, kpad, strip, row_step;
+    if (!vec || (t.rank > 8 && t.Ufrag == nullptr)) {
+      path = PATH_GENERIC; kpad = 0; strip = 64; row_step = 1;
+    } else if (t.rank <= 8) {
+      path = PATH_FMA; kpad = t.rank <= 4 ? 4 : 8; strip = 256; row_step = 1;
+    } else {
+      path = PATH_MMA; kpad = t.rank <= 16 ? 16 : (t.rank <= 32 ? 32 : 64);
+      strip = mma_strip_cols(kpad); row_step = mma_rows_per_iter(kpad);
+    }
+    (void)eb;
+    Group& g = group_for(path, t.dtype, kpad);
+    for (int64_t c0 = 0; c0 < t.cols; c0 += strip) {
+      const int ncols = static_cast<int>(std::min<int64_t>(strip, t.cols - c0));
+      int64_t nrows = std::max<int64_t>(1, target / ncols);
+      nrows = ((nrows + row_step - 1) / row_step) * row_step;
+      // even out the chunks of this strip
+      const int64_t n_chunks = (t.rows + nrows - 1) / nrows;
+      nrows = (t.rows + n_chunks - 1) / n_chunks;
+      nrows = ((nrows + row_step - 1) / row_step) * row_step;
+      for (int64_t r0 = 0; r0 < t.rows; r0 += nrows)
+        g.items.push_back(WorkItem{l, ncols, r0, std::min(nrows, t.rows - r0), c0});
+    }
+  }
+  for (Group& g : out) g.grid = static_cast<int>(std::min<int64_t>(static_cast<int64_t>(g.items.size()), static_cast<int64_t>(sm_count) * blocks_per_sm(g.kc.path)));
+}
+
+int check(zgr_ctx* ctx, cudaError_t e) {
+  if (e == cudaSuccess) return ZGR_OK;
+  const int code = (e == cudaErrorMemoryAllocation) ? ZGR_ENOMEM : ZGR_ECUDA;
+  if (ctx && ctx->sticky == 0) ctx->sticky = code;
+  return code;
+}
+
+template <typename T>
+int dev_alloc(zgr_ctx* ctx, T** p, size_t count) {
+  void* q = nullptr;
+  const int rc = check(ctx, cudaMalloc(&q, std::max<size_t>(count, 1) * sizeof(T)));
+  if (rc != ZGR_OK) return rc;
+  ctx->owned.push_back(q);
+  *p = static_cast<T*>(q);
+  return ZGR_OK;
+}
+
+int upload_groups(zgr_ctx* ctx, std::vector<Group>& groups) {
+  for (Group& g : groups) {
+    if (g.items.empty()) continue;
+    int rc = dev_alloc(ctx, &g.d_items, g.items.size());
+    if (rc != ZGR_OK) return rc;
+    rc = check(ctx, cudaMemcpy(g.d_items, g.items.data(), g.items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
+    if (rc != ZGR_OK) return rc;
+  }
+  return ZGR_OK;
+}
+
+// One sweep  theta <- rnd(theta + c z(seed))  over the planned groups.
+int sweep(zgr_ctx* ctx, const std::vector<Group>& groups, const TensorDesc* d_descs, uint64_t seed, double c, cudaStream_t st) {
+  SweepParams p;
+  p.keys = make_keys(seed);
+  p.iso = make_scale(c * ctx->a, ctx->cfg.bits_per_normal);
+  p.unit = make_scale(1.0, ctx->cfg.bits_per_normal);
+  p.tensors = d_descs;
+  p.cb = static_cast<float>(c * ctx->b);
+  p.stats = nullptr;
+  for (const Group& g : groups) {
+    if (g.items.empty()) continue;
+    p.items = g.d_items;
+    p.n_items = static_cast<int32_t>(g.items.size());
+    const int rc = check(ctx, launch_sweep(g.kc, p, g.grid, st));
+    if (rc != ZGR_OK) return rc;
+    ctx->launches++;
+  }
+  return ZGR_OK;
+}
+
+int flush_descs(zgr_ctx* ctx, cudaStream_t st) {
+  if (!ctx->descs_dirty) return ZGR_OK;
+  const int rc = check(ctx, cudaMemcpyAsync(ctx->d_descs, ctx->descs.data(), ctx->descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice, st));
+  if (rc == ZGR_OK) ctx->descs_dirty = false;
+  return rc;
+}
+
+bool is_finite(double x) { return std::isfinite(x); }
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+extern "C" {
+
+int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_config* cfg) {
+  if (!out) return ZGR_EINVAL;
+  *out = nullptr;
+  if (!tensors || !cfg || n <= 0) return ZGR_EINVAL;
+  if (!(cfg->alpha >= 0.0 && cfg->alpha <= 1.0) || !is_finite(cfg->eps) || !(cfg->eps > 0.0)) return ZGR_EINVAL;
+  if (cfg->scale_mode != ZGR_SCALE_PAPER && cfg->scale_mode != ZGR_SCALE_UNIT) return ZGR_EINVAL;
+  if (cfg->bits_per_normal != 32 && cfg->bits_per_normal != 16) return ZGR_EINVAL;
+  int64_t d = 0, K = 0;
+  for (int32_t l = 0; l < n; ++l) {
+    const zgr_tensor& t = tensors[l];
+    if (!t.data || t.rows < 1 || t.cols < 1) return ZGR_EINVAL;
+    if (t.dtype != ZGR_F32 && t.dtype != ZGR_F16 && t.dtype != ZGR_BF16) return ZGR_EINVAL;
+    if (t.rank < 0 || t.rank > ZGR_MAX_RANK) return ZGR_EINVAL;
+    if ((t.rank == 0) != (t.U == nullptr)) return ZGR_EINVAL;
+    if (reinterpret_cast<uintptr_t>(t.data) % dtype_bytes(t.dtype) != 0) return ZGR_EINVAL;
+    if (t.U && reinterpret_cast<uintptr_t>(t.U) % 4 != 0) return ZGR_EINVAL;
+    if (t.rows > (INT64_MAX / t.cols)) return ZGR_EINVAL;
+    d += t.rows * t.cols;
+    K += static_cast<int64_t>(t.rank) * t.cols;
+  }
+
+  zgr_ctx* ctx = new (std::nothrow) zgr_ctx();
+  if (!ctx) return ZGR_ENOMEM;
+  ctx->cfg = *cfg;
+  ctx->d = d;
+  ctx->K = K;
+  // Eq. (perturbation) with n := d and m := K
+  ctx->a = std::sqrt(cfg->alpha / static_cast<double>(d));
+  ctx->b = K > 0 ? std::sqrt((1.0 - cfg->alpha) / static_cast<double>(K)) : 0.0;
+  if (cfg->scale_mode == ZGR_SCALE_UNIT) {
+    ctx->a *= std::sqrt(static_cast<double>(d));
+    ctx->b *= std::sqrt(static_cast<double>(d));
+  }
+
+  int rc = check(ctx, cudaGetDevice(&ctx->device));
+  if (rc == ZGR_OK) rc = check(ctx, cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device));
+  if (rc != ZGR_OK) {
+    delete ctx;
+    return rc;
+  }
+
+  ctx->descs.resize(static_cast<size_t>(n));
+  const bool guided_on = ctx->b != 0.0;
+  for (int32_t l = 0; l < n && rc == ZGR_OK; ++l) {
+    const zgr_tensor& t = tensors[l];
+    TensorDesc& td = ctx->descs[static_cast<size_t>(l)];
+    td.data = t.data;
+    td.U = t.U;
+    td.Ufrag = nullptr;
+    td.q = nullptr;
+    td.qscale = nullptr;
+    td.qzero = nullptr;
+    td.rows = t.rows;
+    td.cols = t.cols;
+    td.rank = t.rank;
+    td.kpad = 0;
+    td.id = l;
+    td.dtype = t.dtype;
+    const bool vec = (reinterpret_cast<uintptr_t>(t.data) & 15) == 0 && (t.cols % 8 == 0);
+    if (guided_on && t.rank > 8 && vec) {
+      // tensor-core path: library-owned copy of U in A-fragment order
+      td.kpad = t.rank <= 16 ? 16 : (t.rank <= 32 ? 32 : 64);
+      const int64_t tiles = (t.rows + 15) / 16;
+      const size_t n_frag = static_cast<size_t>(tiles) * (td.kpad / 16) * 2 * 32;
+      uint4* frag = nullptr;
+      rc = dev_alloc(ctx, &frag, n_frag);
+      if (rc == ZGR_OK) rc = check(ctx, launch_split_subspace(t.U, t.rows, t.rank, td.kpad, frag, nullptr));
+      if (rc == ZGR_OK) ctx->launches++;
+      td.Ufrag = frag;
+    }
+  }
+  if (rc == ZGR_OK) rc = dev_alloc(ctx, &ctx->d_descs, ctx->descs.size());
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(ctx->d_descs, ctx->descs.data(), ctx->descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+  if (rc == ZGR_OK) {
+    std::vector<int> all(static_cast<size_t>(n));
+    for (int32_t l = 0; l < n; ++l) all[static_cast<size_t>(l)] = l;
+    plan(ctx->descs, all, guided_on, cfg->bits_per_normal, ctx->sm_count, ctx->groups);
+    rc = upload_groups(ctx, ctx->groups);
+  }
+  if (rc == ZGR_OK) rc = dev_alloc(ctx, &ctx->d_stats, static_cast<size_t>(3 * n));
+  if (rc == ZGR_OK) rc = check(ctx, cudaDeviceSynchronize());  // the subspace copies are complete
+  if (rc != ZGR_OK) {
+    zgr_destroy(ctx);
+    return rc;
+  }
+  ctx->sticky = 0;
+  *out = ctx;
+  return ZGR_OK;
+}
+
+int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream) {
+  if (!ctx || !is_finite(scale)) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (ctx->active && ctx->seed != seed) return ZGR_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = flush_descs(ctx, st);
+  if (rc != ZGR_OK) return rc;
+  rc = sweep(ctx, ctx->groups, ctx->d_descs, seed, scale, st);
+  if (rc != ZGR_OK) return rc;
+  ctx->active = true;
+  ctx->seed = seed;
+  ctx->net += scale;
+  return ZGR_OK;
+}
+
+int zgr_restore_update(zgr_ctx* ctx, uint64_t seed, double loss_plus, double loss_minus, double lr, void* stream) {
+  if (!ctx || !is_finite(loss_plus) || !is_finite(loss_minus) || !is_finite(lr)) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (!ctx->active || ctx->seed != seed) return ZGR_ESTATE;
+  // Eq. (grad): projected gradient; Algorithm 1 "Update": W <- W - eta g z, fused with the restore
+  const double g = (loss_plus - loss_minus) / (2.0 * ctx->cfg.eps);
+  const double c = -ctx->net - lr * g;
+  if (!is_finite(c)) return ZGR_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = flush_descs(ctx, st);
+  if (rc != ZGR_OK) return rc;
+  rc = sweep(ctx, ctx->groups, ctx->d_descs, seed, c, st);
+  if (rc != ZGR_OK) return rc;
+  ctx->active = false;
+  ctx->net = 0.0;
+  return ZGR_OK;
+}
+
+int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits) {
+  if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
+  if (!q || !scale || bits != 8) return ZGR_EINVAL;
+  TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
+  if (td.rank == 0) return ZGR_EINVAL;
+  if (ctx->active) return ZGR_ESTATE;
+  td.q = q;
+  td.qscale = scale;
+  td.qzero = zero;
+  ctx->descs_dirty = true;
+  return ZGR_OK;
+}
+
+int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor) {
+  if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
+  TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
+  if (td.rank == 0) return ZGR_EINVAL;
+  if (ctx->active) return ZGR_ESTATE;
+  td.q = nullptr;
+  td.qscale = nullptr;
+  td.qzero = nullptr;
+  ctx->descs_dirty = true;
+  return ZGR_OK;
+}
+
+int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
+  if (!ctx || !out) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = flush_descs(ctx, st);
+  if (rc != ZGR_OK) return rc;
+  const size_t n = ctx->descs.size();
+  if (ctx->stats_items.empty()) {
+    // generic tiling of every tensor: strips of 64 columns
+    int64_t total = ctx->d;
+    int64_t target = std::min<int64_t>(std::max<int64_t>(total / (static_cast<int64_t>(ctx->sm_count) * 64), 4096), 131072);
+    for (size_t l = 0; l < n; ++l) {
+      const TensorDesc& t = ctx->descs[l];
+      for (int64_t c0 = 0; c0 < t.cols; c0 += 64) {
+        const int ncols = static_cast<int>(std::min<int64_t>(64, t.cols - c0));
+        const int64_t nrows = std::max<int64_t>(1, target / ncols);
+        for (int64_t r0 = 0; r0 < t.rows; r0 += nrows)
+          ctx->stats_items.push_back(WorkItem{static_cast<int32_t>(l), ncols, r0, std::min(nrows, t.rows - r0), c0});
+      }
+    }
+    rc = dev_alloc(ctx, &ctx->d_stats_items, ctx->stats_items.size());
+    if (rc == ZGR_OK)
+      rc = check(ctx, cudaMemcpy(ctx->d_stats_items, ctx->stats_items.data(), ctx->stats_items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
+    if (rc != ZGR_OK) return rc;
+  }
+  rc = check(ctx, cudaMemsetAsync(ctx->d_stats, 0, 3 * n * sizeof(double), st));
+  if (rc != ZGR_OK) return rc;
+  SweepParams p;
+  p.keys = make_keys(seed);
+  p.iso = make_scale(ctx->a, ctx->cfg.bits_per_normal);
+  p.unit = make_scale(1.0, ctx->cfg.bits_per_normal);
+  p.tensors = ctx->d_descs;
+  p.items = ctx->d_stats_items;
+  p.n_items = static_cast<int32_t>(ctx->stats_items.size());
+  p.cb = static_cast<float>(ctx->b);
+  p.stats = ctx->d_stats;
+  const int grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * 4));
+  rc = check(ctx, launch_stats(ctx->cfg.bits_per_normal, p, grid, st));
+  if (rc != ZGR_OK) return rc;
+  ctx->launches++;
+  rc = check(ctx, cudaMemcpyAsync(out, ctx->d_stats, 3 * n * sizeof(double), cudaMemcpyDeviceToHost, st));
+  if (rc != ZGR_OK) return rc;
+  return check(ctx, cudaStreamSynchronize(st));
+}
+
+int zgr_debug_philox(zgr_ctx* ctx, uint64_t seed, int32_t tensor, int32_t tag, uint64_t first_block, int64_t n_blocks, uint32_t* dev_out,
+                     void* stream) {
+  if (!ctx || !dev_out || n_blocks < 0 || tensor < 0 || tag < 0) return ZGR_EINVAL;
+  if (reinterpret_cast<uintptr_t>(dev_out) % 16 != 0) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (n_blocks == 0) return ZGR_OK;
+  const int rc = check(ctx, launch_philox_blocks(make_keys(seed), static_cast<uint32_t>(tensor), static_cast<uint32_t>(tag), first_block, n_blocks,
+                                                 dev_out, static_cast<cudaStream_t>(stream)));
+  if (rc == ZGR_OK) ctx->launches++;
+  return rc;
+}
+
+int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, void* stream) {
+  if (!ctx || !dev_out || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
+  if (reinterpret_cast<uintptr_t>(dev_out) % 4 != 0) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // a one-tensor model whose weights are the zeroed output buffer, swept once with scale 1
+  std::vector<TensorDesc> one(1, ctx->descs[static_cast<size_t>(tensor)]);
+  one[0].data = dev_out;
+  one[0].dtype = ZGR_F32;
+  std::vector<Group> groups;
+  const bool guided_on = ctx->b != 0.0;
+  plan(one, std::vector<int>(1, 0), guided_on, ctx->cfg.bits_per_normal, ctx->sm_count, groups);
+  const size_t owned_before = ctx->owned.size();
+  TensorDesc* d_one = nullptr;
+  int rc = dev_alloc(ctx, &d_one, 1);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(d_one, one.data(), sizeof(TensorDesc), cudaMemcpyHostToDevice));
+  if (rc == ZGR_OK) rc = upload_groups(ctx, groups);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemsetAsync(dev_out, 0, static_cast<size_t>(one[0].rows * one[0].cols) * sizeof(float), st));
+  if (rc == ZGR_OK) rc = sweep(ctx, groups, d_one, seed, 1.0, st);
+  if (rc == ZGR_OK) rc = check(ctx, cudaStreamSynchronize(st));
+  for (size_t i = owned_before; i < ctx->owned.size(); ++i) cudaFree(ctx->owned[i]);
+  ctx->owned.resize(owned_before);
+  return rc;
+}
+
+int zgr_get_scalars(const zgr_ctx* ctx, double* a, double* b) {
+  if (!ctx || !a || !b) return ZGR_EINVAL;
+  *a = ctx->a;
+  *b = ctx->b;
+  return ZGR_OK;
+}
+
+int zgr_get_state(const zgr_ctx* ctx, int32_t* active, uint64_t* seed, double* net_scale) {
+  if (!ctx || !active || !seed || !net_scale) return ZGR_EINVAL;
+  *active = ctx->active ? 1 : 0;
+  *seed = ctx->seed;
+  *net_scale = ctx->net;
+  return ZGR_OK;
+}
+
+int64_t zgr_launch_count(const zgr_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+void zgr_destroy(zgr_ctx* ctx) {
+  if (!ctx) return;
+  for (void* p : ctx->owned) cudaFree(p);
+  delete ctx;
+}
+
+const char* zgr_strerror(int code) {
+  switch (code) {
+    case ZGR_OK: return "ok";
+    case ZGR_EINVAL: return "invalid argument";
+    case ZGR_ESTATE: return "call out of sequence (perturb / restore_update seeds do not match)";
+    case ZGR_ECUDA: return "CUDA runtime error (no device, launch failure); the context is unusable";
+    case ZGR_ENOMEM: return "out of device or host memory";
+    default: return "unknown error code";
+  }
+}
+
+}  // extern "C"

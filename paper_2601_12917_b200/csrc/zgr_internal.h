@@ -1,0 +1,63 @@
+// Structures shared by the host side of the library and its kernels.
+#ifndef ZGR_INTERNAL_H_
+#define ZGR_INTERNAL_H_
+
+#include <stdint.h>
+
+namespace zgr {
+
+// Device-side description of one weight tensor.
+struct TensorDesc {
+  void* data;            // weights, rows x cols, row-major
+  const float* U;        // rows x rank fp32 (caller's), or null
+  const uint4* Ufrag;    // library-owned copy of U, split into bf16 hi/lo and laid out in the
+                         // register order of the m16n8k16 A operand (tensor-core path only)
+  const int8_t* q;       // DTC codes rank x cols, or null -> coefficients drawn from the seed
+  const float* qscale;   // rank
+  const float* qzero;    // rank or null
+  int64_t rows, cols;
+  int32_t rank;          // r
+  int32_t kpad;          // r rounded up to the contraction width of the path in use
+  int32_t id;            // generator tensor id (third counter word)
+  int32_t dtype;
+};
+
+// One unit of work of a sweep kernel.
+//   flat items (isotropic kernel): elements [e0, e0 + count) of the tensor, e0 a multiple of 8
+//   tile items (guided kernels):   rows [row0, row0 + nrows) x columns [col0, col0 + ncols)
+struct WorkItem {
+  int32_t tensor;        // index into the descriptor table
+  int32_t ncols;
+  int64_t row0_or_e0;
+  int64_t nrows_or_count;
+  int64_t col0;
+};
+
+// Round keys of Philox4x32-10 for one seed: the key bumped by the Weyl constants once per round.
+struct PhiloxKeys {
+  uint32_t k0[10];
+  uint32_t k1[10];
+};
+
+// Constants of the Gaussian transform with an output scale s folded in (see box_muller()).
+struct NormalScale {
+  float kr;       // -2 ln(2) s^2      : rho'^2 = kr * log2(u1)
+  float s2;       // s^2               : used by the accurate radius near u1 -> 1
+  float phase;    // 2 pi (2^-(nb+1) - 1) - 2 pi   (s >= 0)   or   ... - pi   (s < 0)
+  float u1_off;   // 2^-(nb+1) - 1
+};
+
+// Per-launch constants (passed by value in the kernel parameter space).
+struct SweepParams {
+  PhiloxKeys keys;
+  NormalScale iso;       // isotropic normals, scaled by c*a
+  NormalScale unit;      // coefficient normals, unscaled
+  const TensorDesc* tensors;
+  const WorkItem* items;
+  int32_t n_items;
+  float cb;              // c * b : coefficient of U G
+  double* stats;         // 3 doubles per tensor (stats kernels only)
+};
+
+}  // namespace zgr
+#endif  // ZGR_INTERNAL_H_

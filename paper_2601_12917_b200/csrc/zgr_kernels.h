@@ -1,0 +1,33 @@
+// Host-visible launchers of the sweep kernels.
+#ifndef ZGR_KERNELS_H_
+#define ZGR_KERNELS_H_
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "zgr_internal.h"
+
+namespace zgr {
+
+enum Path { PATH_ISO = 0, PATH_FMA = 1, PATH_MMA = 2, PATH_GENERIC = 3, PATH_COUNT = 4 };
+
+// Which kernel instantiation a group of work items runs on.
+struct KernelChoice {
+  int path;   // Path
+  int dtype;  // ZGR_F32 | ZGR_F16 | ZGR_BF16
+  int kpad;   // FMA: 4 or 8;  MMA: 16, 32 or 64;  otherwise 0
+  int bits;   // 32 or 16 random bits per normal
+};
+
+int mma_strip_cols(int kpad);     // columns of a CTA strip on the tensor-core path
+int mma_rows_per_iter(int kpad);  // rows a CTA advances per iteration there
+size_t mma_smem_bytes(int kpad);
+
+cudaError_t launch_sweep(const KernelChoice& kc, const SweepParams& p, int grid, cudaStream_t st);
+cudaError_t launch_stats(int bits, const SweepParams& p, int grid, cudaStream_t st);
+cudaError_t launch_split_subspace(const float* U, int64_t rows, int r, int kp, uint4* out, cudaStream_t st);
+cudaError_t launch_philox_blocks(const PhiloxKeys& keys, uint32_t tensor, uint32_t tag, uint64_t first_block, int64_t n_blocks,
+                                 uint32_t* out, cudaStream_t st);
+
+}  // namespace zgr
+#endif  // ZGR_KERNELS_H_

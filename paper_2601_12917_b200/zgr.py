@@ -1,0 +1,194 @@
+"""ctypes binding of the ZGR C ABI (``include/zgr.h``).
+
+Argument marshalling only: every step of the path (generator, Gaussian transform, ``U G``
+synthesis, the in-place sweeps, the norm bookkeeping) runs in the CUDA library.  torch tensors
+are used for device memory and streams; the library sees raw pointers.  If ``libzgr.so`` is
+missing the import of the library fails loudly -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libzgr.so")
+
+OK, EINVAL, ESTATE, ECUDA, ENOMEM = 0, -1, -2, -3, -4
+F32, F16, BF16 = 0, 1, 2
+SCALE_PAPER, SCALE_UNIT = 0, 1
+TAG_ISO, TAG_COEFF = 0, 1
+MAX_RANK = 64
+
+
+class ZgrTensor(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("dtype", ctypes.c_int32),
+                ("rank", ctypes.c_int32), ("U", ctypes.c_void_p)]
+
+
+class ZgrConfig(ctypes.Structure):
+    _fields_ = [("alpha", ctypes.c_double), ("eps", ctypes.c_double), ("scale_mode", ctypes.c_int32), ("bits_per_normal", ctypes.c_int32)]
+
+
+class ZgrError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libzgr.so`` (built in-tree by ``paper_2601_12917_b200/build.py``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_12917_b200.build` "
+                              "(there is no CPU fallback for the ZGR step)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, u64, dbl = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64, ctypes.c_double
+        L.zgr_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(ZgrTensor), i32, ctypes.POINTER(ZgrConfig)]
+        L.zgr_perturb.argtypes = [vp, u64, dbl, vp]
+        L.zgr_restore_update.argtypes = [vp, u64, dbl, dbl, dbl, vp]
+        L.zgr_set_coeffs_dtc.argtypes = [vp, i32, vp, vp, vp, i32]
+        L.zgr_clear_coeffs.argtypes = [vp, i32]
+        L.zgr_get_stats.argtypes = [vp, u64, ctypes.POINTER(dbl), vp]
+        L.zgr_debug_philox.argtypes = [vp, u64, i32, i32, u64, i64, vp, vp]
+        L.zgr_debug_z.argtypes = [vp, u64, i32, vp, vp]
+        L.zgr_get_scalars.argtypes = [vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+        L.zgr_get_state.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(u64), ctypes.POINTER(dbl)]
+        L.zgr_launch_count.argtypes = [vp]
+        L.zgr_launch_count.restype = i64
+        L.zgr_destroy.argtypes = [vp]
+        L.zgr_destroy.restype = None
+        L.zgr_strerror.argtypes = [ctypes.c_int]
+        L.zgr_strerror.restype = ctypes.c_char_p
+        for name in ("zgr_init", "zgr_perturb", "zgr_restore_update", "zgr_set_coeffs_dtc", "zgr_clear_coeffs", "zgr_get_stats",
+                     "zgr_debug_philox", "zgr_debug_z", "zgr_get_scalars", "zgr_get_state"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().zgr_strerror(code).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != OK:
+        raise ZgrError(code, what)
+
+
+def _dtype_code(t) -> int:
+    import torch
+    return {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}[t.dtype]
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class Zgr:
+    """A ZGR context over a list of device tensors (``zgr_init`` ... ``zgr_destroy``).
+
+    ``weights[l]`` is a contiguous CUDA tensor (1-D or 2-D; fp32, fp16 or bf16) updated in place;
+    ``subspaces[l]`` is ``None`` or a contiguous fp32 CUDA tensor of shape (rows, rank) with
+    orthonormal columns.  The context keeps references to all of them.
+    """
+
+    def __init__(self, weights: Sequence, subspaces: Sequence, alpha: float, eps: float, scale_mode: int = SCALE_UNIT,
+                 bits_per_normal: int = 32):
+        assert len(weights) == len(subspaces)
+        self._keep: List = [list(weights), list(subspaces)]
+        n = len(weights)
+        arr = (ZgrTensor * n)()
+        for l, (w, U) in enumerate(zip(weights, subspaces)):
+            if not w.is_cuda or not w.is_contiguous():
+                raise ValueError(f"tensor {l}: weights must be contiguous CUDA tensors")
+            rows, cols = (1, w.numel()) if w.dim() == 1 else (w.shape[0], w.shape[1])
+            rank = 0
+            uptr = None
+            if U is not None:
+                if not U.is_cuda or not U.is_contiguous() or U.shape[0] != rows:
+                    raise ValueError(f"tensor {l}: subspace must be a contiguous CUDA tensor of shape (rows, rank)")
+                rank, uptr = int(U.shape[1]), U.data_ptr()
+            arr[l] = ZgrTensor(w.data_ptr(), rows, cols, _dtype_code(w), rank, uptr)
+        cfg = ZgrConfig(alpha, eps, scale_mode, bits_per_normal)
+        self._h = ctypes.c_void_p()
+        _check(lib().zgr_init(ctypes.byref(self._h), arr, n, ctypes.byref(cfg)), "zgr_init")
+        self.n = n
+
+    # -- the three calls of a step --------------------------------------------------------------
+    def perturb(self, seed: int, scale: float, stream=None) -> None:
+        _check(lib().zgr_perturb(self._h, seed, scale, _stream_ptr(stream)), "zgr_perturb")
+
+    def restore_update(self, seed: int, loss_plus: float, loss_minus: float, lr: float, stream=None) -> None:
+        _check(lib().zgr_restore_update(self._h, seed, loss_plus, loss_minus, lr, _stream_ptr(stream)), "zgr_restore_update")
+
+    # -- compressed coefficients ----------------------------------------------------------------
+    def set_coeffs_dtc(self, tensor: int, q, scale, zero=None, bits: int = 8) -> None:
+        self._keep.append((q, scale, zero))
+        _check(lib().zgr_set_coeffs_dtc(self._h, tensor, q.data_ptr(), scale.data_ptr(), None if zero is None else zero.data_ptr(), bits),
+               "zgr_set_coeffs_dtc")
+
+    def clear_coeffs(self, tensor: int) -> None:
+        _check(lib().zgr_clear_coeffs(self._h, tensor), "zgr_clear_coeffs")
+
+    # -- bookkeeping and test hooks -------------------------------------------------------------
+    def get_stats(self, seed: int, stream=None):
+        import numpy as np
+        out = (ctypes.c_double * (3 * self.n))()
+        _check(lib().zgr_get_stats(self._h, seed, out, _stream_ptr(stream)), "zgr_get_stats")
+        return np.ctypeslib.as_array(out).reshape(self.n, 3).copy()
+
+    def debug_philox(self, seed: int, tensor: int, tag: int, first_block: int, n_blocks: int, stream=None):
+        import torch
+        out = torch.empty((n_blocks, 4), dtype=torch.int32, device="cuda")
+        _check(lib().zgr_debug_philox(self._h, seed, tensor, tag, first_block, n_blocks, out.data_ptr(), _stream_ptr(stream)), "zgr_debug_philox")
+        return out
+
+    def debug_z(self, seed: int, tensor: int, stream=None):
+        import torch
+        w = self._keep[0][tensor]
+        out = torch.empty(w.shape, dtype=torch.float32, device=w.device)
+        _check(lib().zgr_debug_z(self._h, seed, tensor, out.data_ptr(), _stream_ptr(stream)), "zgr_debug_z")
+        return out
+
+    def scalars(self):
+        a, b = ctypes.c_double(), ctypes.c_double()
+        _check(lib().zgr_get_scalars(self._h, ctypes.byref(a), ctypes.byref(b)), "zgr_get_scalars")
+        return a.value, b.value
+
+    def state(self):
+        act, seed, net = ctypes.c_int32(), ctypes.c_uint64(), ctypes.c_double()
+        _check(lib().zgr_get_state(self._h, ctypes.byref(act), ctypes.byref(seed), ctypes.byref(net)), "zgr_get_state")
+        return bool(act.value), seed.value, net.value
+
+    def launch_count(self) -> int:
+        return int(lib().zgr_launch_count(self._h))
+
+    def close(self) -> None:
+        if self._h:
+            lib().zgr_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def from_device_model(dm, bits_per_normal: int = 32) -> Zgr:
+    """Context over a :class:`synth.DeviceModel`, with its DTC payloads attached if it has any."""
+    wl = dm.workload
+    z = Zgr(dm.theta, dm.U, wl.alpha, wl.eps, wl.scale_mode, bits_per_normal)
+    if wl.dtc:
+        for l, q in enumerate(dm.q):
+            if q is not None:
+                z.set_coeffs_dtc(l, q, dm.scale[l])
+    return z

@@ -1,0 +1,127 @@
+"""Shared plumbing of the GPU parity tests: moving tensors between torch (device), the oracle's
+numpy storage and doubles, and the tolerance checks.
+
+Tolerances (stated by the benchmark spec, derived in the design notes):
+  * generator blocks: bit-exact;
+  * fp32 weights: max |gpu - oracle| <= 1e-6 * max|theta| per call;
+  * fp16 / bf16 weights: |gpu - oracle| <= 1 ulp of the storage type per call, the ulp taken at the
+    larger of |theta before| and |theta after| (where theta + c z cancels, the ulp of the tiny
+    result is below the resolution of the fp32 arithmetic both operands went through).
+Each check also reports how many elements moved at all, so that a sweep that does nothing cannot pass.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2601_12917_b200 import synth, zgr
+
+TORCH_DTYPE = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
+ORACLE_DTYPE = {"f32": oracle.F32, "f16": oracle.F16, "bf16": oracle.BF16}
+SIG_BITS = {"f32": 24, "f16": 11, "bf16": 8}
+EMIN = {"f32": -126, "f16": -14, "bf16": -126}
+
+
+def to_storage(t: torch.Tensor) -> np.ndarray:
+    """Device tensor -> the oracle's storage array (float32, or uint16 bit patterns)."""
+    t = t.detach().contiguous()
+    if t.dtype == torch.float32:
+        return t.cpu().numpy().reshape(-1).copy()
+    return t.view(torch.int16).cpu().numpy().view(np.uint16).reshape(-1).copy()
+
+
+def to_double(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy().reshape(-1)
+
+
+def from_double(x: np.ndarray, dtype: str, shape, device) -> torch.Tensor:
+    """Doubles that are exactly representable in `dtype` -> device tensor."""
+    return torch.from_numpy(np.asarray(x, dtype=np.float64)).to(TORCH_DTYPE[dtype]).reshape(shape).to(device)
+
+
+def ulp(x: np.ndarray, dtype: str) -> np.ndarray:
+    ax = np.maximum(np.abs(x), 2.0 ** EMIN[dtype])
+    return 2.0 ** (np.floor(np.log2(ax)) - (SIG_BITS[dtype] - 1))
+
+
+def check_sweep(got: np.ndarray, exp: np.ndarray, before: np.ndarray, dtype: str, theta_max: float, what: str = "") -> dict:
+    """Assert the per-call tolerance; returns a small report."""
+    diff = np.abs(got - exp)
+    if dtype == "f32":
+        tol = 1e-6 * theta_max
+        worst = float(diff.max()) if diff.size else 0.0
+        assert worst <= tol, f"{what}: fp32 max-abs error {worst:.3e} > {tol:.3e}"
+    else:
+        u = ulp(np.maximum(np.abs(before), np.abs(exp)), dtype)
+        bad = diff > u
+        assert not bad.any(), (f"{what}: {int(bad.sum())} of {bad.size} elements differ by more than 1 ulp; "
+                               f"worst {float((diff / u).max()):.2f} ulp")
+    return {"equal": float(np.mean(got == exp)) if got.size else 1.0, "moved": float(np.mean(exp != before)) if got.size else 0.0,
+            "max_abs": float(diff.max()) if diff.size else 0.0}
+
+
+class Pair:
+    """The same small model on both sides: device tensors for the library, storage arrays for the oracle."""
+
+    def __init__(self, shapes, ranks, dtype: str, alpha=0.5, eps=1e-3, scale_mode=zgr.SCALE_UNIT, bits=32, seed=0, device="cuda",
+                 dtc=None, misalign=False):
+        self.dtype, self.device, self.bits = dtype, device, bits
+        self.shapes, self.ranks = list(shapes), list(ranks)
+        self.theta, self.U, self.q, self.scale, self.zero = [], [], [], [], []
+        for l, ((m, n), r) in enumerate(zip(shapes, ranks)):
+            w = oracle.round_to(synth.weights_host(synth.TensorSpec(f"t{l}", m, n, r), seed + l).ravel(), ORACLE_DTYPE[dtype])
+            if misalign:
+                # view into a larger buffer, offset by one element: not 16-byte aligned
+                buf = torch.zeros(m * n + 1, dtype=TORCH_DTYPE[dtype], device=device)
+                t = buf[1:].view(m, n) if m > 1 else buf[1:]
+                t.copy_(from_double(w, dtype, t.shape, device))
+                self.theta.append(t)
+            else:
+                self.theta.append(from_double(w, dtype, (m, n) if m > 1 else (n,), device))
+            self.U.append(torch.from_numpy(synth.subspace(m, r, seed * 1000 + l)).to(device) if r > 0 else None)
+            self.q.append(None); self.scale.append(None); self.zero.append(None)
+        self.lib = zgr.Zgr(self.theta, self.U, alpha, eps, scale_mode, bits)
+        self.alpha, self.eps, self.scale_mode = alpha, eps, scale_mode
+        self.d = sum(m * n for m, n in shapes)
+        self.K = sum(r * n for (m, n), r in zip(shapes, ranks))
+        self.a, self.b = oracle.mix_scalars(alpha, self.d, self.K, scale_mode)
+        self.theta_max = max(float(t.abs().max()) for t in self.theta)
+
+    def set_dtc(self, l: int, q: np.ndarray, scale: np.ndarray, zero=None):
+        self.q[l] = torch.from_numpy(q).to(self.device)
+        self.scale[l] = torch.from_numpy(scale).to(self.device)
+        self.zero[l] = None if zero is None else torch.from_numpy(zero).to(self.device)
+        self.lib.set_coeffs_dtc(l, self.q[l], self.scale[l], self.zero[l])
+
+    def oracle_tensor(self, l: int) -> oracle.OracleTensor:
+        (m, n) = self.shapes[l]
+        U = None if self.U[l] is None else self.U[l].cpu().numpy()
+        q = None if self.q[l] is None else self.q[l].cpu().numpy()
+        sc = None if self.scale[l] is None else self.scale[l].cpu().numpy()
+        ze = None if self.zero[l] is None else self.zero[l].cpu().numpy()
+        return oracle.OracleTensor(theta=to_storage(self.theta[l]), rows=m, cols=n, dtype=ORACLE_DTYPE[self.dtype], U=U, q=q, scale=sc, zero=ze)
+
+    def call_and_check(self, seed: int, c: float, fn, what: str):
+        """Run one library call `fn()` that applies coefficient c; the oracle starts from the same theta."""
+        ots = [self.oracle_tensor(l) for l in range(len(self.shapes))]
+        before = [oracle.decode(t.theta, t.dtype) for t in ots]
+        fn()
+        torch.cuda.synchronize()
+        reports = []
+        for l, t in enumerate(ots):
+            oracle.sweep_tensor(t, seed, l, self.bits, self.a, self.b, c)
+            exp = oracle.decode(t.theta, t.dtype)
+            got = to_double(self.theta[l])
+            reports.append(check_sweep(got, exp, before[l], self.dtype, self.theta_max, f"{what} tensor {l} {self.shapes[l]} r={self.ranks[l]}"))
+        return reports
+
+    def step(self, seed: int, lp: float, lm: float, lr: float):
+        """perturb(+eps), perturb(-2 eps), restore_update, each checked against the oracle."""
+        eps = self.eps
+        r1 = self.call_and_check(seed, eps, lambda: self.lib.perturb(seed, eps), "perturb(+eps)")
+        r2 = self.call_and_check(seed, -2 * eps, lambda: self.lib.perturb(seed, -2 * eps), "perturb(-2eps)")
+        g = oracle.projected_grad(lp, lm, eps)
+        c = eps - lr * g
+        r3 = self.call_and_check(seed, c, lambda: self.lib.restore_update(seed, lp, lm, lr), "restore_update")
+        return r1, r2, r3
