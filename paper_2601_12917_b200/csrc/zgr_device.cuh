@@ -67,24 +67,30 @@ __device__ __forceinline__ float cos_approx(float x) {
 }
 
 // m1, m2: the two uniform fields already placed in mantissa position (bits 0..22).
-// PRECISE selects a radius that stays accurate where u1 is close to 1: the hardware log2 has an
-// absolute error of about 2^-22 there, which the square root would amplify for the smallest radii;
-// for 1 - u1 < 2^-6 the series -2 ln(1-v) = 2v + v^2 + (2/3) v^3 is used instead.  fp32 weights
-// need it for their 1e-6 tolerance; 16-bit weights do not.
+//
+// PRECISE = false (16-bit weights): hardware log2 / sqrt / sin / cos approximations; absolute error of
+// a unit normal about 4e-6, far below one ulp of the storage type times any step coefficient.
+// PRECISE = true (fp32 weights, tolerance 1e-6 max|theta|): logf, correctly rounded sqrtf and
+// sincospif on the exactly representable angle 2 u2 (in units of pi), a few fp32 ulp in total.
+// The fast form cannot serve fp32: besides the sin/cos error, the hardware log2 has an absolute
+// error near 2^-22 for u1 close to 1, which the square root amplifies for the smallest radii.
 template <bool PRECISE>
 __device__ __forceinline__ void box_muller(uint32_t m1, uint32_t m2, const NormalScale& ns, float& n0, float& n1) {
   const float u1 = __uint_as_float(0x3F800000u | m1) + ns.u1_off;
   const float t2 = __uint_as_float(0x3F800000u | m2);
-  float r2 = fabsf(ns.kr * lg2_approx(u1));
   if (PRECISE) {
-    const float v = 1.0f - u1;
-    const float series = v * fmaf(v, fmaf(v, 0.66666667f, 1.0f), 2.0f) * ns.s2;
-    r2 = v < 0.015625f ? series : r2;
+    const float x = fmaf(2.0f, t2, 2.0f * ns.u1_off);   // 2 u2, exact
+    float sn, cs;
+    sincospif(x, &sn, &cs);
+    const float rho = ns.s * sqrtf(-2.0f * logf(u1));
+    n0 = rho * cs;
+    n1 = rho * sn;
+  } else {
+    const float rho = sqrt_approx(fabsf(ns.kr * lg2_approx(u1)));
+    const float phi = fmaf(t2, 6.28318530717958647692f, ns.phase);
+    n0 = rho * cos_approx(phi);
+    n1 = rho * sin_approx(phi);
   }
-  const float rho = sqrt_approx(r2);
-  const float phi = fmaf(t2, 6.28318530717958647692f, ns.phase);
-  n0 = rho * cos_approx(phi);
-  n1 = rho * sin_approx(phi);
 }
 
 // Eight consecutive normals of stream (tensor, tag) starting at element e (a multiple of 8), each

@@ -70,7 +70,7 @@ NormalScale make_scale(double s, int bits) {
   const double off = std::ldexp(1.0, -(nb + 1)) - 1.0;
   NormalScale ns;
   ns.kr = static_cast<float>(-2.0 * std::log(2.0) * s * s);
-  ns.s2 = static_cast<float>(s * s);
+  ns.s = static_cast<float>(s);
   ns.phase = static_cast<float>(kTwoPi * off + (s >= 0 ? -kTwoPi : -0.5 * kTwoPi));
   ns.u1_off = static_cast<float>(off);
   return ns;
@@ -85,8 +85,11 @@ int blocks_per_sm(int path) {
 }
 
 // Split the tensors listed in `which` into work items, grouped by the kernel that serves them.
+// The kernel family follows the tensor's own storage type (fp32 tensors take the accurate transform and
+// an exact fp32 contraction); `kernel_dtype` >= 0 overrides only the type the kernel reads and writes,
+// which lets the test hook run a 16-bit tensor's kernel family on an fp32 image.
 void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, bool guided_on, int bits, int sm_count,
-          std::vector<Group>& out) {
+          std::vector<Group>& out, int kernel_dtype = -1) {
   int64_t total = 0;
   for (int l : which) total += descs[l].rows * descs[l].cols;
   // elements per item: enough items for ~16 rounds over the resident CTAs, but large enough that the
@@ -94,14 +97,16 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
   int64_t target = total / (static_cast<int64_t>(sm_count) * 2 * 16);
   target = std::min<int64_t>(std::max<int64_t>(target, 16384), 524288);
 
-  std::map<std::tuple<int, int, int>, size_t> index;  // (path, dtype, kpad) -> group
-  auto group_for = [&](int path, int dtype, int kpad) -> Group& {
-    auto key = std::make_tuple(path, dtype, kpad);
+  std::map<std::tuple<int, int, int, int>, size_t> index;  // (path, dtype, kpad, precise) -> group
+  auto group_for = [&](int path, int real_dtype, int kpad) -> Group& {
+    const int precise = real_dtype == ZGR_F32 ? 1 : 0;
+    const int dtype = kernel_dtype >= 0 ? kernel_dtype : real_dtype;
+    auto key = std::make_tuple(path, dtype, kpad, precise);
     auto it = index.find(key);
     if (it == index.end()) {
       index[key] = out.size();
       Group g;
-      g.kc = KernelChoice{path, dtype, kpad, bits};
+      g.kc = KernelChoice{path, dtype, kpad, bits, precise};
       out.push_back(std::move(g));
       return out.back();
     }
@@ -110,7 +115,6 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
 
   for (int l : which) {
     const TensorDesc& t = descs[l];
-    const int eb = dtype_bytes(t.dtype);
     const bool aligned = (reinterpret_cast<uintptr_t>(t.data) & 15) == 0;
     const bool guided = guided_on && t.rank > 0;
     if (!guided) {
@@ -131,7 +135,6 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
       path = PATH_MMA; kpad = t.rank <= 16 ? 16 : (t.rank <= 32 ? 32 : 64);
       strip = mma_strip_cols(kpad); row_step = mma_rows_per_iter(kpad);
     }
-    (void)eb;
     Group& g = group_for(path, t.dtype, kpad);
     for (int64_t c0 = 0; c0 < t.cols; c0 += strip) {
       const int ncols = static_cast<int>(std::min<int64_t>(strip, t.cols - c0));
@@ -269,7 +272,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
     td.id = l;
     td.dtype = t.dtype;
     const bool vec = (reinterpret_cast<uintptr_t>(t.data) & 15) == 0 && (t.cols % 8 == 0);
-    if (guided_on && t.rank > 8 && vec) {
+    if (guided_on && t.rank > 8 && vec && t.dtype != ZGR_F32) {
       // tensor-core path: library-owned copy of U in A-fragment order
       td.kpad = t.rank <= 16 ? 16 : (t.rank <= 32 ? 32 : 64);
       const int64_t tiles = (t.rows + 15) / 16;
@@ -423,10 +426,9 @@ int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, voi
   // a one-tensor model whose weights are the zeroed output buffer, swept once with scale 1
   std::vector<TensorDesc> one(1, ctx->descs[static_cast<size_t>(tensor)]);
   one[0].data = dev_out;
-  one[0].dtype = ZGR_F32;
   std::vector<Group> groups;
   const bool guided_on = ctx->b != 0.0;
-  plan(one, std::vector<int>(1, 0), guided_on, ctx->cfg.bits_per_normal, ctx->sm_count, groups);
+  plan(one, std::vector<int>(1, 0), guided_on, ctx->cfg.bits_per_normal, ctx->sm_count, groups, ZGR_F32);
   const size_t owned_before = ctx->owned.size();
   TensorDesc* d_one = nullptr;
   int rc = dev_alloc(ctx, &d_one, 1);

@@ -42,7 +42,7 @@ struct PhiloxKeys {
 // Constants of the Gaussian transform with an output scale s folded in (see box_muller()).
 struct NormalScale {
   float kr;       // -2 ln(2) s^2      : rho'^2 = kr * log2(u1)
-  float s2;       // s^2               : used by the accurate radius near u1 -> 1
+  float s;        // the scale itself (accurate transform)
   float phase;    // 2 pi (2^-(nb+1) - 1) - 2 pi   (s >= 0)   or   ... - pi   (s < 0)
   float u1_off;   // 2^-(nb+1) - 1
 };

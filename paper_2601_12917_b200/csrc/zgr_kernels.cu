@@ -434,19 +434,23 @@ cudaError_t launch_typed(const KernelChoice& kc, const SweepParams& p, int grid,
       sweep_generic_kernel<T, BITS, PRECISE><<<grid, kThreads, 0, st>>>(p);
       break;
     case PATH_MMA: {
-      const size_t smem = mma_smem_bytes(kc.kpad);
-      if (kc.kpad == 16) {
-        auto k = sweep_mma_kernel<T, BITS, PRECISE, 16, 1>;
-        cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        k<<<grid, kThreads, smem, st>>>(p);
-      } else if (kc.kpad == 32) {
-        auto k = sweep_mma_kernel<T, BITS, PRECISE, 32, 1>;
-        cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        k<<<grid, kThreads, smem, st>>>(p);
+      if constexpr (PRECISE) {
+        return cudaErrorInvalidValue;  // the split-bf16 contraction cannot meet the fp32 tolerance
       } else {
-        auto k = sweep_mma_kernel<T, BITS, PRECISE, 64, 2>;
-        cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        k<<<grid, kThreads, smem, st>>>(p);
+        const size_t smem = mma_smem_bytes(kc.kpad);
+        if (kc.kpad == 16) {
+          auto k = sweep_mma_kernel<T, BITS, false, 16, 1>;
+          cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+          k<<<grid, kThreads, smem, st>>>(p);
+        } else if (kc.kpad == 32) {
+          auto k = sweep_mma_kernel<T, BITS, false, 32, 1>;
+          cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+          k<<<grid, kThreads, smem, st>>>(p);
+        } else {
+          auto k = sweep_mma_kernel<T, BITS, false, 64, 2>;
+          cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+          k<<<grid, kThreads, smem, st>>>(p);
+        }
       }
       break;
     }
@@ -458,9 +462,16 @@ cudaError_t launch_typed(const KernelChoice& kc, const SweepParams& p, int grid,
 
 template <typename T>
 cudaError_t launch_dtype(const KernelChoice& kc, const SweepParams& p, int grid, cudaStream_t st) {
-  constexpr bool precise = sizeof(T) == 4;
-  if (kc.bits == 32) return launch_typed<T, 32, precise>(kc, p, grid, st);
-  return launch_typed<T, 16, precise>(kc, p, grid, st);
+  if (kc.precise) {
+    if constexpr (sizeof(T) == 4) {
+      if (kc.bits == 32) return launch_typed<T, 32, true>(kc, p, grid, st);
+      return launch_typed<T, 16, true>(kc, p, grid, st);
+    } else {
+      return cudaErrorInvalidValue;  // 16-bit storage never needs the accurate transform
+    }
+  }
+  if (kc.bits == 32) return launch_typed<T, 32, false>(kc, p, grid, st);
+  return launch_typed<T, 16, false>(kc, p, grid, st);
 }
 
 }  // namespace

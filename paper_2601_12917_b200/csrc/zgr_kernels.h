@@ -17,6 +17,7 @@ struct KernelChoice {
   int dtype;  // ZGR_F32 | ZGR_F16 | ZGR_BF16
   int kpad;   // FMA: 4 or 8;  MMA: 16, 32 or 64;  otherwise 0
   int bits;   // 32 or 16 random bits per normal
+  int precise;  // accurate Gaussian transform (tensors stored in fp32)
 };
 
 int mma_strip_cols(int kpad);     // columns of a CTA strip on the tensor-core path

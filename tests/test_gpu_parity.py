@@ -38,32 +38,38 @@ def test_generator_many_blocks():
 
 # ------------------------------------------------------------------------------------- z itself
 Z_CASES = [
-    # (shape, rank, tolerance on z, what it exercises)
-    ((1, 1000), 0, 1e-5, "iso vector + ragged tail"),
-    ((64, 256), 4, 1e-5, "fma R=4"),
-    ((300, 520), 8, 1e-5, "fma R=8, three strips, last one ragged"),
-    ((37, 264), 3, 1e-5, "fma rank 3 padded to 4"),
-    ((50, 72), 5, 1e-5, "fma rank 5 padded to 8"),
-    ((100, 1032), 16, 1e-4, "mma K=16, ragged strip and row tile"),
-    ((130, 512), 32, 1e-4, "mma K=32"),
-    ((96, 520), 64, 1e-4, "mma K=64"),
-    ((48, 128), 12, 1e-4, "mma rank 12 padded to 16"),
-    ((33, 64), 40, 1e-4, "mma rank 40 padded to 64"),
-    ((45, 100), 6, 1e-5, "generic (columns not a multiple of 8), low rank"),
-    ((45, 100), 20, 1e-5, "generic, high rank"),
+    # (shape, rank, kernel family of 16-bit tensors, what it exercises)
+    ((1, 1000), 0, "iso", "iso vector + ragged tail"),
+    ((64, 256), 4, "fma", "fma R=4"),
+    ((300, 520), 8, "fma", "fma R=8, three strips, last one ragged"),
+    ((37, 264), 3, "fma", "fma rank 3 padded to 4"),
+    ((50, 72), 5, "fma", "fma rank 5 padded to 8"),
+    ((100, 1032), 16, "mma", "mma K=16, ragged strip and row tile"),
+    ((130, 512), 32, "mma", "mma K=32"),
+    ((96, 520), 64, "mma", "mma K=64"),
+    ((48, 128), 12, "mma", "mma rank 12 padded to 16"),
+    ((72, 64), 40, "mma", "mma rank 40 padded to 64"),
+    ((45, 100), 6, "generic", "generic (columns not a multiple of 8), low rank"),
+    ((45, 100), 20, "generic", "generic, high rank"),
 ]
+# absolute tolerance on a unit-variance z: fp32 tensors use the accurate transform and an exact fp32
+# contraction; 16-bit tensors use the hardware approximations and, above rank 8, split-bf16 tensor cores
+Z_TOL = {("f32", "iso"): 2e-6, ("f32", "fma"): 2e-6, ("f32", "mma"): 3e-6, ("f32", "generic"): 3e-6,
+         ("bf16", "iso"): 1e-5, ("bf16", "fma"): 1e-5, ("bf16", "mma"): 1e-4, ("bf16", "generic"): 1e-5}
 
 
 @pytest.mark.parametrize("bits", [32, 16])
-@pytest.mark.parametrize("shape,rank,tol,what", Z_CASES)
-def test_perturbation_matches_oracle(shape, rank, tol, what, bits):
-    p = Pair([shape, (1, 40)], [rank, 0], "f32", bits=bits, seed=3)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape,rank,family,what", Z_CASES)
+def test_perturbation_matches_oracle(shape, rank, family, what, dtype, bits):
+    p = Pair([shape, (1, 40)], [rank, 0], dtype, bits=bits, seed=3)
     seed = 1234567
+    tol = Z_TOL[(dtype, family)]
     for l in range(2):
         got = to_double(p.lib.debug_z(seed, l))
         exp = oracle.z_tensor(p.oracle_tensor(l), seed, l, bits, p.a, p.b).ravel()
         err = np.abs(got - exp).max()
-        assert err <= tol, f"{what}: max |z_gpu - z_oracle| = {err:.3e}"
+        assert err <= tol, f"{what} [{dtype}]: max |z_gpu - z_oracle| = {err:.3e}"
         assert np.abs(exp).max() > 0.5
 
 
@@ -71,7 +77,7 @@ def test_perturbation_matches_oracle(shape, rank, tol, what, bits):
 @pytest.mark.parametrize("alpha", [0.0, 0.3, 1.0])
 def test_perturbation_scalings_and_alpha_limits(scale_mode, alpha):
     shapes, ranks = [(64, 256), (1, 64), (64, 128)], [8, 0, 16]
-    p = Pair(shapes, ranks, "f32", alpha=alpha, scale_mode=scale_mode)
+    p = Pair(shapes, ranks, "bf16", alpha=alpha, scale_mode=scale_mode)
     a, b = p.lib.scalars()
     assert a == pytest.approx(p.a, rel=1e-14) and b == pytest.approx(p.b, rel=1e-14, abs=1e-300)
     for l in range(3):
@@ -103,7 +109,8 @@ def test_step_per_call_parity(model, dtype, bits):
     for call in reports:
         for rep in call:
             assert rep["moved"] > 0.3, rep         # the sweep really changed the weights
-            assert rep["equal"] > 0.9, rep         # and almost every element is bit-identical to the oracle
+            if dtype != "f32":
+                assert rep["equal"] > 0.9, rep     # and almost every 16-bit result is bit-identical to the oracle
     assert p.lib.state()[0] is False
 
 
