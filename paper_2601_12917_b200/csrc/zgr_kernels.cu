@@ -115,10 +115,10 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_con
         normals8<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso, z);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          float acc = th[i] + z[i];
+          float acc = z[i];  // the perturbation is summed on its own scale, then added to theta once
 #pragma unroll
           for (int k = 0; k < R; ++k) acc = fmaf(u[k], g[k][i], acc);
-          th[i] = acc;
+          th[i] += acc;
         }
         Storage<T>::store8(base + e, th);
       }
@@ -149,9 +149,9 @@ __global__ void __launch_bounds__(kThreads) sweep_generic_kernel(const __grid_co
     const int64_t row_end = w.row0_or_e0 + w.nrows_or_count;
     for (int64_t row = w.row0_or_e0 + rg; row < row_end; row += kThreads / 64) {
       const int64_t e = row * td.cols + w.col0 + cl;
-      float acc = Storage<T>::load1(base + e) + normal1<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso);
+      float acc = normal1<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso);
       for (int k = 0; k < r; ++k) acc = fmaf(__ldg(td.U + row * r + k), Gs[k][cl], acc);
-      Storage<T>::store1(base + e, acc);
+      Storage<T>::store1(base + e, Storage<T>::load1(base + e) + acc);
     }
   }
 }
