@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the ZGR step on synthetic LLaMA-7B-shaped bf16 parameters (one B200 per process).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama_7b] [--bits 16|32]
+    python bench.py --impl reference ...        # the CPU oracle on a bounded sample, same JSON line
+
+A "step" is the whole hot path once: for each of the Q perturbation queries of the workload,
+perturb(+eps), perturb(-2 eps), restore_update(lr/Q) -- 3Q in-place sweeps over every weight tensor.
+`value` = model parameters stepped per second (parameters x steps / time, all ranks), measured with
+CUDA events with weights, subspaces and work tables resident in HBM.  `e2e` repeats the measurement
+with the per-step inputs coming from the host through the C ABI: every guided tensor's subspace is
+copied from pinned host memory (zgr_update_subspace), the step runs, and the per-tensor norms are read
+back to the host (zgr_get_stats).  The weights themselves stay in HBM in both: keeping the model on
+the device and never materialising z is the point of the method.
+
+The path does not shard (one GPU holds the model; the only cross-rank quantities would be two loss
+scalars), so --gpus N runs N independent replicas and reports their sum ("replicas only").
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "zgr_step_params_per_sec"
+UNIT = "params/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------ oracle legs
+def oracle_sample(wl, rows: int, sweeps: int, bits: int):
+    """Time `sweeps` oracle sweeps over a slab (rows x cols of the workload's first attention matrix,
+    with its rank).  Returns (seconds, elements, threads)."""
+    import numpy as np
+    import oracle
+    from paper_2601_12917_b200 import synth
+    spec = next(t for t in wl.tensors if t.rank > 0 and t.rows == t.cols)
+    rows = min(rows, spec.rows)
+    dt = {"f32": oracle.F32, "f16": oracle.F16, "bf16": oracle.BF16}[wl.dtype]
+    w = synth.weights_host(synth.TensorSpec("slab", rows, spec.cols, spec.rank), 0).ravel()
+    U = synth.subspace(rows, spec.rank, 0)
+    q = sc = None
+    if wl.dtc:
+        q, sc = synth.dtc_payload(spec.rank, spec.cols, 0)
+    t = oracle.OracleTensor(theta=oracle.encode(w, dt), rows=rows, cols=spec.cols, dtype=dt, U=U, q=q, scale=sc)
+    a, b = oracle.mix_scalars(wl.alpha, wl.params, wl.coeffs, wl.scale_mode)
+    coeff = [wl.eps, -2 * wl.eps, wl.eps]
+    t0 = time.perf_counter()
+    for s in range(sweeps):
+        oracle.sweep_tensor(t, 1 + s // 3, 1, bits, a, b, coeff[s % 3])
+    return time.perf_counter() - t0, rows * spec.cols, oracle.num_threads(), f"{rows}x{spec.cols} slab of a rank-{spec.rank} {wl.dtype} matrix"
+
+
+def cpu_baseline(wl, bits: int):
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample of the workload."""
+    import oracle
+    oracle.build()
+    rows = (1 << 26) // 4096 if wl.params > (1 << 28) else 2048
+    secs, n, threads, what = oracle_sample(wl, rows, 1, bits)
+    sweeps_per_step = 3 * wl.queries
+    return {"value": n / secs / sweeps_per_step, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"one sweep over a {what}, scaled by 1/{sweeps_per_step} sweeps per step ({secs:.2f} s)"}
+
+
+def run_reference(args, wl):
+    """`--impl reference`: the CPU oracle, K steps of 3Q sweeps over a bounded slab."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    sweeps_per_step = 3 * wl.queries
+    rows = 1024
+    for _ in range(args.warmup):
+        oracle_sample(wl, 64, 1, args.bits)
+    t0 = time.perf_counter()
+    total = 0.0
+    n = 0
+    for _ in range(args.steps):
+        secs, n, threads, what = oracle_sample(wl, rows, sweeps_per_step, args.bits)
+        total += secs
+    value = n * args.steps / total
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": wl.name, "sample": what, "queries": wl.queries, "bits_per_normal": args.bits},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": f"{args.steps} steps of {sweeps_per_step} sweeps over a {what}"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    def __init__(self, index):
+        self.path = f"/tmp/zgr_clocks_{os.getpid()}.csv"
+        self.proc = None
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+                 "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for ln in open(self.path):
+                parts = [x.strip() for x in ln.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0])); mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, parts[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def reduce_over_ranks(ms_local: float, units_local: float, dist=None):
+    """(max over ranks of the elapsed time, sum over ranks of the units processed)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return ms_local, units_local
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def run_step(z, wl, t: int):
+    for q in range(wl.queries):
+        seed = wl.seed(t, q)
+        lp, lm = wl.losses(t, q)
+        z.perturb(seed, wl.eps)
+        z.perturb(seed, -2.0 * wl.eps)
+        z.restore_update(seed, lp, lm, wl.lr / wl.queries)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="zgr", choices=["zgr", "reference"])
+    ap.add_argument("--workload", default="llama_7b")
+    ap.add_argument("--layers", type=int, default=None, help="shrink the model (profiling captures only)")
+    ap.add_argument("--bits", type=int, default=16, choices=[16, 32], help="random bits per normal")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    from paper_2601_12917_b200 import synth
+    wl = synth.workload(args.workload, layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(wl, args.bits)        # before the first CUDA call
+
+    import torch
+    import torch.distributed as dist
+    from paper_2601_12917_b200 import zgr
+    zgr.lib()                                     # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    device = torch.device("cuda", local_rank)
+
+    dm = synth.materialise(wl, device, seed=rank)
+    z = zgr.from_device_model(dm, args.bits)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        run_step(z, wl, t)
+    barrier()
+
+    # ---- timed region: K steps, device-resident inputs ----
+    cvd = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
+    sampler = ClockSampler(cvd[local_rank] if local_rank < len(cvd) else local_rank)
+    time.sleep(0.3)
+    launches0 = z.launch_count()
+    z.profile(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for t in range(args.steps):
+        run_step(z, wl, args.warmup + t)
+    ev1.record(stream)
+    barrier()
+    ms_local = ev0.elapsed_time(ev1)
+    kernels = z.profile_read()
+    z.profile(False)
+    launches = z.launch_count() - launches0
+    clocks = sampler.stop()
+    ms, units = reduce_over_ranks(ms_local, float(wl.params) * args.steps, dist if world > 1 else None)
+    value = units / (ms * 1e-3)
+
+    # ---- roofline of the dominant kernel ----
+    peak, peak_kind = load_peaks()
+    eb = synth.DTYPE_BYTES[wl.dtype]
+    top = max(kernels, key=lambda k: k["ms_total"]) if kernels else None
+    roofline = None
+    if top:
+        per_launch_ms = top["ms_total"] / top["launches"]
+        achieved = 2 * eb * top["elements"] / (per_launch_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                    "peak_kind": f"of {peak_kind}", "kernel": f"sweep_{top['path']}_kernel(k={top['kpad']})", "launches": top["launches"],
+                    "ms_per_launch": per_launch_ms, "algorithmic_bytes_per_launch": 2 * eb * top["elements"],
+                    "share_of_kernel_time": top["ms_total"] / sum(k["ms_total"] for k in kernels)}
+
+    # ---- end to end: per-step inputs from pinned host memory, result read back ----
+    e2e = None
+    if not args.no_e2e:
+        guided = [l for l, U in enumerate(dm.U) if U is not None]
+        host_U = {l: dm.U[l].cpu().pin_memory() for l in guided}
+        h2d = sum(h.numel() * 4 for h in host_U.values())
+        d2h = 3 * 8 * len(dm.theta)
+        n_e2e = max(1, min(args.steps, 3))
+
+        def e2e_step(t):
+            for l in guided:
+                z.update_subspace(l, host_U[l])
+            run_step(z, wl, t)
+            return z.get_stats(wl.seed(t, 0))
+
+        e2e_step(10_000)
+        barrier()
+        ev0.record(stream)
+        for t in range(n_e2e):
+            e2e_step(20_000 + t)
+        ev1.record(stream)
+        barrier()
+        ms_e, units_e = reduce_over_ranks(ev0.elapsed_time(ev1), float(wl.params) * n_e2e, dist if world > 1 else None)
+        e2e = {"value": units_e / (ms_e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
+               "ms_per_step": ms_e / n_e2e, "what": "subspaces H2D from pinned memory + step + per-tensor norms D2H, through the C ABI"}
+
+    if rank == 0:
+        sweeps = 3 * wl.queries
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic",
+                "config": {"workload": wl.name, "storage": wl.dtype, "params": wl.params, "tensors": len(wl.tensors), "rank": wl.rank,
+                           "queries": wl.queries, "sweeps_per_step": sweeps, "bits_per_normal": args.bits, "alpha": wl.alpha, "eps": wl.eps,
+                           "lr": wl.lr, "scale_mode": "unit", "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only"},
+                "sweep_params_per_s": value * sweeps, "hbm_gbs_all_sweeps": value * sweeps * 2 * eb / 1e9,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
+                "kernels": kernels}
+        print(json.dumps(line), flush=True)
+    z.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

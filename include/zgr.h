@@ -110,6 +110,15 @@ int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const floa
 /* Back to seed-drawn coefficients for `tensor` (Algorithm 1, "Sample z_g").  Errors as above. */
 int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor);
 
+/* A guided round delivers a new subspace for `tensor` (Algorithm 1, "Collect gradients to build basis
+ * V_r", transmitted layer by layer as in Sec. 3.3).  U_src: rows x rank fp32 row-major, on the host
+ * (src_is_host != 0; pinned memory makes the copy asynchronous) or on the device, or NULL if the caller
+ * has already rewritten the device buffer given to zgr_init in place.  The values are copied into that
+ * device buffer (it is overwritten) on `stream`, and the library's own operand copy of U for the
+ * tensor-core kernels is rebuilt.  ZGR_EINVAL: bad index or tensor without subspace.
+ * ZGR_ESTATE: a perturbation is active. */
+int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_t src_is_host, void* stream);
+
 /* Norm bookkeeping for the adaptive choice of alpha mentioned in Sec. 1: for each tensor l,
  * out[3l+0] = sum (a Z_l)^2, out[3l+1] = sum (b U_l G_l)^2, out[3l+2] = sum z_l^2 for `seed`.
  * Reads no weights.  `out` is a HOST array of 3*n doubles; the call synchronises `stream`. */
@@ -122,6 +131,18 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream);
 int zgr_debug_philox(zgr_ctx* ctx, uint64_t seed, int32_t tensor, int32_t tag, uint64_t first_block, int64_t n_blocks,
                      uint32_t* dev_out, void* stream);
 int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, void* stream);
+
+/* Per-kernel timing.  While enabled, every sweep launch is bracketed by CUDA events on its stream.
+ * zgr_profile_read synchronises the device, writes one entry per kernel family that ran since the
+ * last read (up to max_entries) and clears the record.  path: 0 isotropic, 1 CUDA-core rank<=8,
+ * 2 tensor-core, 3 fallback; elements = weights covered by one launch. */
+typedef struct {
+  int32_t path, dtype, kpad, launches;
+  int64_t elements;
+  double ms_total;
+} zgr_kernel_time;
+int zgr_profile(zgr_ctx* ctx, int32_t enable);
+int zgr_profile_read(zgr_ctx* ctx, zgr_kernel_time* out, int32_t max_entries, int32_t* n_entries);
 
 /* Introspection: mixing scalars a, b in double; active seed / net scale (active = 0 when idle);
  * number of kernel launches issued by this context so far. */

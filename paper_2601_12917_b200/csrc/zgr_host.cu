@@ -23,6 +23,8 @@ struct Group {
   std::vector<WorkItem> items;
   WorkItem* d_items = nullptr;
   int grid = 0;
+  int64_t elements = 0;                                   // weights covered by one launch
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed;  // per-launch events while profiling is on
 };
 
 int dtype_bytes(int dt) { return dt == ZGR_F32 ? 4 : 2; }
@@ -48,6 +50,7 @@ struct zgr_ctx {
   double net = 0;
   int sticky = 0;                     // first CUDA failure, returned by every later call
   int64_t launches = 0;
+  bool profiling = false;
 };
 
 namespace {
@@ -148,6 +151,10 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
         g.items.push_back(WorkItem{l, ncols, r0, std::min(nrows, t.rows - r0), c0});
     }
   }
+  for (Group& g : out) {
+    g.elements = 0;
+    for (const WorkItem& w : g.items) g.elements += g.kc.path == PATH_ISO ? w.nrows_or_count : w.nrows_or_count * w.ncols;
+  }
   for (Group& g : out) g.grid = static_cast<int>(std::min<int64_t>(static_cast<int64_t>(g.items.size()), static_cast<int64_t>(sm_count) * blocks_per_sm(g.kc.path)));
 }
 
@@ -180,7 +187,7 @@ int upload_groups(zgr_ctx* ctx, std::vector<Group>& groups) {
 }
 
 // One sweep  theta <- rnd(theta + c z(seed))  over the planned groups.
-int sweep(zgr_ctx* ctx, const std::vector<Group>& groups, const TensorDesc* d_descs, uint64_t seed, double c, cudaStream_t st) {
+int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, uint64_t seed, double c, cudaStream_t st) {
   SweepParams p;
   p.keys = make_keys(seed);
   p.iso = make_scale(c * ctx->a, ctx->cfg.bits_per_normal);
@@ -188,12 +195,21 @@ int sweep(zgr_ctx* ctx, const std::vector<Group>& groups, const TensorDesc* d_de
   p.tensors = d_descs;
   p.cb = static_cast<float>(c * ctx->b);
   p.stats = nullptr;
-  for (const Group& g : groups) {
+  for (Group& g : groups) {
     if (g.items.empty()) continue;
     p.items = g.d_items;
     p.n_items = static_cast<int32_t>(g.items.size());
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (ctx->profiling) {
+      if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return check(ctx, cudaErrorUnknown);
+      cudaEventRecord(e0, st);
+    }
     const int rc = check(ctx, launch_sweep(g.kc, p, g.grid, st));
     if (rc != ZGR_OK) return rc;
+    if (ctx->profiling) {
+      cudaEventRecord(e1, st);
+      g.timed.emplace_back(e0, e1);
+    }
     ctx->launches++;
   }
   return ZGR_OK;
@@ -442,6 +458,63 @@ int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, voi
   return rc;
 }
 
+int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_t src_is_host, void* stream) {
+  if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
+  TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
+  if (td.rank == 0) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (ctx->active) return ZGR_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = ZGR_OK;
+  if (U_src != nullptr && U_src != td.U) {
+    const size_t bytes = static_cast<size_t>(td.rows) * td.rank * sizeof(float);
+    rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.U), U_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, st));
+    if (rc != ZGR_OK) return rc;
+  }
+  if (td.Ufrag != nullptr) {
+    rc = check(ctx, launch_split_subspace(td.U, td.rows, td.rank, td.kpad, const_cast<uint4*>(td.Ufrag), st));
+    if (rc == ZGR_OK) ctx->launches++;
+  }
+  return rc;
+}
+
+int zgr_profile(zgr_ctx* ctx, int32_t enable) {
+  if (!ctx) return ZGR_EINVAL;
+  ctx->profiling = enable != 0;
+  return ZGR_OK;
+}
+
+int zgr_profile_read(zgr_ctx* ctx, zgr_kernel_time* out, int32_t max_entries, int32_t* n_entries) {
+  if (!ctx || !out || !n_entries || max_entries < 0) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  const int rc = check(ctx, cudaDeviceSynchronize());
+  if (rc != ZGR_OK) return rc;
+  int32_t n = 0;
+  for (Group& g : ctx->groups) {
+    if (g.timed.empty()) continue;
+    double total = 0.0;
+    for (auto& ev : g.timed) {
+      float ms = 0.0f;
+      if (cudaEventElapsedTime(&ms, ev.first, ev.second) == cudaSuccess) total += ms;
+      cudaEventDestroy(ev.first);
+      cudaEventDestroy(ev.second);
+    }
+    if (n < max_entries) {
+      zgr_kernel_time& o = out[n];
+      o.path = g.kc.path;
+      o.dtype = g.kc.dtype;
+      o.kpad = g.kc.kpad;
+      o.launches = static_cast<int32_t>(g.timed.size());
+      o.elements = g.elements;
+      o.ms_total = total;
+      ++n;
+    }
+    g.timed.clear();
+  }
+  *n_entries = n;
+  return ZGR_OK;
+}
+
 int zgr_get_scalars(const zgr_ctx* ctx, double* a, double* b) {
   if (!ctx || !a || !b) return ZGR_EINVAL;
   *a = ctx->a;
@@ -461,6 +534,11 @@ int64_t zgr_launch_count(const zgr_ctx* ctx) { return ctx ? ctx->launches : -1; 
 
 void zgr_destroy(zgr_ctx* ctx) {
   if (!ctx) return;
+  for (Group& g : ctx->groups)
+    for (auto& ev : g.timed) {
+      cudaEventDestroy(ev.first);
+      cudaEventDestroy(ev.second);
+    }
   for (void* p : ctx->owned) cudaFree(p);
   delete ctx;
 }

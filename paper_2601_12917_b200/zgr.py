@@ -30,6 +30,14 @@ class ZgrConfig(ctypes.Structure):
     _fields_ = [("alpha", ctypes.c_double), ("eps", ctypes.c_double), ("scale_mode", ctypes.c_int32), ("bits_per_normal", ctypes.c_int32)]
 
 
+class ZgrKernelTime(ctypes.Structure):
+    _fields_ = [("path", ctypes.c_int32), ("dtype", ctypes.c_int32), ("kpad", ctypes.c_int32), ("launches", ctypes.c_int32),
+                ("elements", ctypes.c_int64), ("ms_total", ctypes.c_double)]
+
+
+PATH_NAMES = {0: "iso", 1: "fma", 2: "mma", 3: "generic"}
+
+
 class ZgrError(RuntimeError):
     def __init__(self, code: int, what: str):
         super().__init__(f"{what}: {strerror(code)} ({code})")
@@ -58,6 +66,9 @@ def lib() -> ctypes.CDLL:
         L.zgr_debug_z.argtypes = [vp, u64, i32, vp, vp]
         L.zgr_get_scalars.argtypes = [vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
         L.zgr_get_state.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(u64), ctypes.POINTER(dbl)]
+        L.zgr_update_subspace.argtypes = [vp, i32, vp, i32, vp]
+        L.zgr_profile.argtypes = [vp, i32]
+        L.zgr_profile_read.argtypes = [vp, ctypes.POINTER(ZgrKernelTime), i32, ctypes.POINTER(i32)]
         L.zgr_launch_count.argtypes = [vp]
         L.zgr_launch_count.restype = i64
         L.zgr_destroy.argtypes = [vp]
@@ -65,7 +76,8 @@ def lib() -> ctypes.CDLL:
         L.zgr_strerror.argtypes = [ctypes.c_int]
         L.zgr_strerror.restype = ctypes.c_char_p
         for name in ("zgr_init", "zgr_perturb", "zgr_restore_update", "zgr_set_coeffs_dtc", "zgr_clear_coeffs", "zgr_get_stats",
-                     "zgr_debug_philox", "zgr_debug_z", "zgr_get_scalars", "zgr_get_state"):
+                     "zgr_debug_philox", "zgr_debug_z", "zgr_get_scalars", "zgr_get_state", "zgr_update_subspace", "zgr_profile",
+                     "zgr_profile_read"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -137,6 +149,26 @@ class Zgr:
 
     def clear_coeffs(self, tensor: int) -> None:
         _check(lib().zgr_clear_coeffs(self._h, tensor), "zgr_clear_coeffs")
+
+    def update_subspace(self, tensor: int, U_src=None, stream=None) -> None:
+        """New subspace for `tensor`: a torch tensor on the host (pinned for an asynchronous copy) or on
+        the device, or None if the device buffer given at construction was rewritten in place."""
+        if U_src is None:
+            ptr, host = None, 0
+        else:
+            assert U_src.is_contiguous() and U_src.dtype == self._keep[1][tensor].dtype and U_src.shape == self._keep[1][tensor].shape
+            ptr, host = U_src.data_ptr(), 0 if U_src.is_cuda else 1
+        _check(lib().zgr_update_subspace(self._h, tensor, ptr, host, _stream_ptr(stream)), "zgr_update_subspace")
+
+    def profile(self, enable: bool) -> None:
+        _check(lib().zgr_profile(self._h, 1 if enable else 0), "zgr_profile")
+
+    def profile_read(self):
+        arr = (ZgrKernelTime * 64)()
+        n = ctypes.c_int32()
+        _check(lib().zgr_profile_read(self._h, arr, 64, ctypes.byref(n)), "zgr_profile_read")
+        return [{"path": PATH_NAMES.get(e.path, str(e.path)), "dtype": e.dtype, "kpad": e.kpad, "launches": e.launches,
+                 "elements": e.elements, "ms_total": e.ms_total} for e in arr[: n.value]]
 
     # -- bookkeeping and test hooks -------------------------------------------------------------
     def get_stats(self, seed: int, stream=None):
