@@ -39,7 +39,7 @@ extern "C" {
 
 #define ZGR_MAX_RANK 64 /* largest subspace rank r per tensor */
 
-enum { ZGR_OK = 0, ZGR_EINVAL = -1, ZGR_ESTATE = -2, ZGR_ECUDA = -3, ZGR_ENOMEM = -4 };
+enum { ZGR_OK = 0, ZGR_EINVAL = -1, ZGR_ESTATE = -2, ZGR_ECUDA = -3, ZGR_ENOMEM = -4, ZGR_ETOOBIG = -5 };
 
 /* storage type of a weight tensor; arithmetic is fp32, one round-to-nearest-even per sweep */
 enum { ZGR_F32 = 0, ZGR_F16 = 1, ZGR_BF16 = 2 };
@@ -123,6 +123,25 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
  * out[3l+0] = sum (a Z_l)^2, out[3l+1] = sum (b U_l G_l)^2, out[3l+2] = sum z_l^2 for `seed`.
  * Reads no weights.  `out` is a HOST array of 3*n doubles; the call synchronises `stream`. */
 int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream);
+
+/* The norms of ONE tensor, computed without allocating anything.  (The paper has no counterpart; this
+ * entry point exists for callers that cannot allocate device memory while they run: loops in which the
+ * device-wide synchronisation implied by cudaMalloc/cudaFree would stall other streams, and processes
+ * whose framework has already claimed all free device memory for its own pool.)
+ * Same three sums as zgr_get_stats for `tensor`, written to dev_out3 (DEVICE, 3 doubles, 8-byte
+ * aligned) by work enqueued on `stream`; the call does not synchronise.  All intermediate storage is a
+ * fixed array inside the library image: 3 * ZGR_NOALLOC_MAX_TILES doubles (192 KiB), resident on every
+ * GPU that loads the library until the process exits.  A tile is 1024 rows x 64 columns, so tensors
+ * up to ZGR_NOALLOC_MAX_TILES tiles (e.g. 32000 x 16384) fit; larger ones are refused with ZGR_ETOOBIG.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that
+ * first call outside any stream capture.  Every call uses the same array: two calls whose kernels can
+ * overlap on the GPU (different streams, different contexts of this library) race on it, so issue
+ * them on one stream or order them yourself.  Nothing has to be cleared between calls (each call
+ * writes every slot it later reads); after a call the array holds that call's partial sums.  The
+ * summation order is fixed, so repeated calls give identical bits.  Calls no cudaMalloc / cudaFree.
+ * ZGR_EINVAL: null or misaligned dev_out3, bad tensor index. */
+#define ZGR_NOALLOC_MAX_TILES 8192
+int zgr_tensor_norms_noalloc(zgr_ctx* ctx, uint64_t seed, int32_t tensor, double* dev_out3, void* stream);
 
 /* Test hooks.  zgr_debug_philox writes n_blocks raw generator blocks (4 uint32 each) of stream
  * (seed, tensor, tag) starting at first_block to dev_out (device).  zgr_debug_z writes z_l(seed) as

@@ -12,6 +12,7 @@
 
 #include "zgr.h"
 #include "zgr_internal.h"
+#include "zgr_host_internal.h"
 #include "zgr_kernels.h"
 
 using namespace zgr;
@@ -225,6 +226,20 @@ int flush_descs(zgr_ctx* ctx, cudaStream_t st) {
 bool is_finite(double x) { return std::isfinite(x); }
 
 }  // namespace
+
+namespace zgr {
+PhiloxKeys host_make_keys(uint64_t seed) { return make_keys(seed); }
+NormalScale host_make_scale(double s, int bits) { return make_scale(s, bits); }
+bool host_ctx_view(const zgr_ctx* ctx, int32_t l, TensorDesc* desc, double* a, double* b, int* bits, int* sticky) {
+  if (!ctx || l < 0 || l >= static_cast<int32_t>(ctx->descs.size())) return false;
+  *desc = ctx->descs[static_cast<size_t>(l)];
+  *a = ctx->a;
+  *b = ctx->b;
+  *bits = ctx->cfg.bits_per_normal;
+  *sticky = ctx->sticky;
+  return true;
+}
+}  // namespace zgr
 
 // ------------------------------------------------------------------------------------------------
 extern "C" {
@@ -550,6 +565,7 @@ const char* zgr_strerror(int code) {
     case ZGR_ESTATE: return "call out of sequence (perturb / restore_update seeds do not match)";
     case ZGR_ECUDA: return "CUDA runtime error (no device, launch failure); the context is unusable";
     case ZGR_ENOMEM: return "out of device or host memory";
+    case ZGR_ETOOBIG: return "tensor larger than the fixed scratch of the allocation-free entry point (ZGR_NOALLOC_MAX_TILES tiles of 1024 x 64)";
     default: return "unknown error code";
   }
 }

@@ -14,7 +14,8 @@ from typing import List, Optional, Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libzgr.so")
 
-OK, EINVAL, ESTATE, ECUDA, ENOMEM = 0, -1, -2, -3, -4
+OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5
+NOALLOC_MAX_TILES = 8192
 F32, F16, BF16 = 0, 1, 2
 SCALE_PAPER, SCALE_UNIT = 0, 1
 TAG_ISO, TAG_COEFF = 0, 1
@@ -69,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.zgr_update_subspace.argtypes = [vp, i32, vp, i32, vp]
         L.zgr_profile.argtypes = [vp, i32]
         L.zgr_profile_read.argtypes = [vp, ctypes.POINTER(ZgrKernelTime), i32, ctypes.POINTER(i32)]
+        L.zgr_tensor_norms_noalloc.argtypes = [vp, u64, i32, vp, vp]
+        L.zgr_tensor_norms_noalloc.restype = ctypes.c_int
         L.zgr_launch_count.argtypes = [vp]
         L.zgr_launch_count.restype = i64
         L.zgr_destroy.argtypes = [vp]
@@ -176,6 +179,11 @@ class Zgr:
         out = (ctypes.c_double * (3 * self.n))()
         _check(lib().zgr_get_stats(self._h, seed, out, _stream_ptr(stream)), "zgr_get_stats")
         return np.ctypeslib.as_array(out).reshape(self.n, 3).copy()
+
+    def tensor_norms_noalloc(self, seed: int, tensor: int, out, stream=None) -> None:
+        """Norms of one tensor into `out` (a CUDA tensor of 3 float64) without any allocation by the
+        library; asynchronous on the stream.  See zgr_tensor_norms_noalloc in zgr.h for the limits."""
+        _check(lib().zgr_tensor_norms_noalloc(self._h, seed, tensor, out.data_ptr(), _stream_ptr(stream)), "zgr_tensor_norms_noalloc")
 
     def debug_philox(self, seed: int, tensor: int, tag: int, first_block: int, n_blocks: int, stream=None):
         import torch
