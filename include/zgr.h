@@ -163,6 +163,13 @@ typedef struct {
 int zgr_profile(zgr_ctx* ctx, int32_t enable);
 int zgr_profile_read(zgr_ctx* ctx, zgr_kernel_time* out, int32_t max_entries, int32_t* n_entries);
 
+/* Device-side health.  The tensor-core sweep waits on hardware barriers (TMA, tensor memory) with a
+ * time limit; a wait that gives up records a non-zero code, abandons the sweep and lets the kernel
+ * exit cleanly instead of hanging the GPU.  This call synchronises the device and returns that code
+ * in *code (0 = healthy).  A non-zero code makes the context unusable (every later call returns
+ * ZGR_ECUDA): the interrupted sweep left the weights partly updated. */
+int zgr_device_status(zgr_ctx* ctx, int32_t* code);
+
 /* Introspection: mixing scalars a, b in double; active seed / net scale (active = 0 when idle);
  * number of kernel launches issued by this context so far. */
 int zgr_get_scalars(const zgr_ctx* ctx, double* a, double* b);

@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
@@ -52,6 +53,9 @@ struct zgr_ctx {
   int sticky = 0;                     // first CUDA failure, returned by every later call
   int64_t launches = 0;
   bool profiling = false;
+  CUtensorMap* d_tmaps = nullptr;     // three per tensor (theta, U hi, U lo); tcgen05 path only
+  std::vector<CUtensorMap> tmaps;     // host mirror
+  int* d_err = nullptr;               // set by a kernel whose bounded wait gave up
 };
 
 namespace {
@@ -80,10 +84,48 @@ NormalScale make_scale(double s, int bits) {
   return ns;
 }
 
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled through the runtime (the library does not link against libcuda).
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 2-D map over a row-major 16-bit matrix (rows x cols, row pitch = cols), box = box_cols x 128 rows,
+// swizzle matching the box's row length in bytes (32, 64 or 128).
+bool make_map_16bit(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int box_cols) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), 128};
+  const cuuint32_t estr[2] = {1, 1};
+  const int row_bytes = box_cols * 2;
+  const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+  return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool umma_wanted() {
+  const char* e = std::getenv("ZGR_TENSOR_PATH");
+  return !(e && std::strcmp(e, "legacy") == 0);
+}
+
 int blocks_per_sm(int path) {
   switch (path) {
     case PATH_ISO: return 6;
     case PATH_GENERIC: return 4;
+    case PATH_UMMA: return 1;
     default: return 2;
   }
 }
@@ -135,6 +177,8 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
       path = PATH_GENERIC; kpad = 0; strip = 64; row_step = 1;
     } else if (t.rank <= 8) {
       path = PATH_FMA; kpad = t.rank <= 4 ? 4 : 8; strip = 256; row_step = 1;
+    } else if (t.umma && kernel_dtype < 0) {
+      path = PATH_UMMA; kpad = t.kpad; strip = umma_strip_cols(kpad); row_step = 128;
     } else {
       path = PATH_MMA; kpad = t.rank <= 16 ? 16 : (t.rank <= 32 ? 32 : 64);
       strip = mma_strip_cols(kpad); row_step = mma_rows_per_iter(kpad);
@@ -142,7 +186,7 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
     Group& g = group_for(path, t.dtype, kpad);
     for (int64_t c0 = 0; c0 < t.cols; c0 += strip) {
       const int ncols = static_cast<int>(std::min<int64_t>(strip, t.cols - c0));
-      int64_t nrows = std::max<int64_t>(1, target / ncols);
+      int64_t nrows = std::max<int64_t>(1, (path == PATH_UMMA ? 2 * target : target) / ncols);
       nrows = ((nrows + row_step - 1) / row_step) * row_step;
       // even out the chunks of this strip
       const int64_t n_chunks = (t.rows + nrows - 1) / nrows;
@@ -205,7 +249,8 @@ int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, u
       if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return check(ctx, cudaErrorUnknown);
       cudaEventRecord(e0, st);
     }
-    const int rc = check(ctx, launch_sweep(g.kc, p, g.grid, st));
+    const int rc = check(ctx, g.kc.path == PATH_UMMA ? launch_sweep_umma(g.kc, p, ctx->d_tmaps, ctx->d_err, g.grid, st)
+                                                     : launch_sweep(g.kc, p, g.grid, st));
     if (rc != ZGR_OK) return rc;
     if (ctx->profiling) {
       cudaEventRecord(e1, st);
@@ -286,6 +331,8 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
   }
 
   ctx->descs.resize(static_cast<size_t>(n));
+  ctx->tmaps.resize(static_cast<size_t>(3 * n));
+  std::memset(ctx->tmaps.data(), 0, ctx->tmaps.size() * sizeof(CUtensorMap));
   const bool guided_on = ctx->b != 0.0;
   for (int32_t l = 0; l < n && rc == ZGR_OK; ++l) {
     const zgr_tensor& t = tensors[l];
@@ -302,6 +349,9 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
     td.kpad = 0;
     td.id = l;
     td.dtype = t.dtype;
+    td.umma = 0;
+    td.Uhi = nullptr;
+    td.Ulo = nullptr;
     const bool vec = (reinterpret_cast<uintptr_t>(t.data) & 15) == 0 && (t.cols % 8 == 0);
     if (guided_on && t.rank > 8 && vec && t.dtype != ZGR_F32) {
       // tensor-core path: library-owned copy of U in A-fragment order
@@ -313,8 +363,30 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
       if (rc == ZGR_OK) rc = check(ctx, launch_split_subspace(t.U, t.rows, t.rank, td.kpad, frag, nullptr));
       if (rc == ZGR_OK) ctx->launches++;
       td.Ufrag = frag;
+      // tcgen05 + TMA path: row-major hi/lo copies of U and three tensor maps
+      if (rc == ZGR_OK && umma_wanted() && encode_tiled_fn() != nullptr && t.rows < (int64_t{1} << 31) - 256 && t.cols < (int64_t{1} << 31) - 256) {
+        const int64_t rows_pad = ((t.rows + 127) / 128) * 128;
+        uint16_t *hi = nullptr, *lo = nullptr;
+        rc = dev_alloc(ctx, &hi, static_cast<size_t>(rows_pad) * td.kpad);
+        if (rc == ZGR_OK) rc = dev_alloc(ctx, &lo, static_cast<size_t>(rows_pad) * td.kpad);
+        if (rc == ZGR_OK) rc = check(ctx, launch_split_subspace_rowmajor(t.U, t.rows, t.rank, td.kpad, rows_pad, hi, lo, nullptr));
+        if (rc == ZGR_OK) {
+          ctx->launches++;
+          CUtensorMap* m = &ctx->tmaps[static_cast<size_t>(3 * l)];
+          if (make_map_16bit(m, t.data, t.rows, t.cols, 64) && make_map_16bit(m + 1, hi, rows_pad, td.kpad, td.kpad) &&
+              make_map_16bit(m + 2, lo, rows_pad, td.kpad, td.kpad)) {
+            td.umma = 1;
+            td.Uhi = hi;
+            td.Ulo = lo;
+          }
+        }
+      }
     }
   }
+  if (rc == ZGR_OK) rc = dev_alloc(ctx, &ctx->d_tmaps, ctx->tmaps.size());
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(ctx->d_tmaps, ctx->tmaps.data(), ctx->tmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
+  if (rc == ZGR_OK) rc = dev_alloc(ctx, &ctx->d_err, 1);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemset(ctx->d_err, 0, sizeof(int)));
   if (rc == ZGR_OK) rc = dev_alloc(ctx, &ctx->d_descs, ctx->descs.size());
   if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(ctx->d_descs, ctx->descs.data(), ctx->descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
   if (rc == ZGR_OK) {
@@ -490,6 +562,11 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
     rc = check(ctx, launch_split_subspace(td.U, td.rows, td.rank, td.kpad, const_cast<uint4*>(td.Ufrag), st));
     if (rc == ZGR_OK) ctx->launches++;
   }
+  if (rc == ZGR_OK && td.umma) {
+    const int64_t rows_pad = ((td.rows + 127) / 128) * 128;
+    rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.Uhi, td.Ulo, st));
+    if (rc == ZGR_OK) ctx->launches++;
+  }
   return rc;
 }
 
@@ -527,6 +604,19 @@ int zgr_profile_read(zgr_ctx* ctx, zgr_kernel_time* out, int32_t max_entries, in
     g.timed.clear();
   }
   *n_entries = n;
+  return ZGR_OK;
+}
+
+int zgr_device_status(zgr_ctx* ctx, int32_t* code) {
+  if (!ctx || !code) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  int rc = check(ctx, cudaDeviceSynchronize());
+  if (rc != ZGR_OK) return rc;
+  int v = 0;
+  rc = check(ctx, cudaMemcpy(&v, ctx->d_err, sizeof(int), cudaMemcpyDeviceToHost));
+  if (rc != ZGR_OK) return rc;
+  *code = v;
+  if (v != 0) ctx->sticky = ZGR_ECUDA;   // a kernel gave up on a wait: its sweep is incomplete, the weights are not trustworthy
   return ZGR_OK;
 }
 

@@ -20,6 +20,9 @@ struct TensorDesc {
   int32_t kpad;          // r rounded up to the contraction width of the path in use
   int32_t id;            // generator tensor id (third counter word)
   int32_t dtype;
+  int32_t umma;          // 1: served by the tcgen05 + TMA kernel (tensor maps and row-major hi/lo copies of U exist)
+  void* Uhi;             // library-owned, rows_pad x kpad bf16 row-major (TMA source), or null
+  void* Ulo;
 };
 
 // One unit of work of a sweep kernel.

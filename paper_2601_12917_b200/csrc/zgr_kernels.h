@@ -2,6 +2,7 @@
 #ifndef ZGR_KERNELS_H_
 #define ZGR_KERNELS_H_
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 
@@ -9,7 +10,7 @@
 
 namespace zgr {
 
-enum Path { PATH_ISO = 0, PATH_FMA = 1, PATH_MMA = 2, PATH_GENERIC = 3, PATH_COUNT = 4 };
+enum Path { PATH_ISO = 0, PATH_FMA = 1, PATH_MMA = 2, PATH_GENERIC = 3, PATH_UMMA = 4, PATH_COUNT = 5 };
 
 // Which kernel instantiation a group of work items runs on.
 struct KernelChoice {
@@ -25,6 +26,12 @@ int mma_rows_per_iter(int kpad);  // rows a CTA advances per iteration there
 size_t mma_smem_bytes(int kpad);
 
 cudaError_t launch_sweep(const KernelChoice& kc, const SweepParams& p, int grid, cudaStream_t st);
+// tcgen05 + TMA sweep (16-bit weights, rank > 8).  tmaps: three tensor maps per tensor (theta, U hi, U lo).
+int umma_strip_cols(int kpad);
+size_t umma_smem_bytes(int kpad);
+cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
+cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st);
+
 cudaError_t launch_stats(int bits, const SweepParams& p, int grid, cudaStream_t st);
 cudaError_t launch_split_subspace(const float* U, int64_t rows, int r, int kp, uint4* out, cudaStream_t st);
 cudaError_t launch_philox_blocks(const PhiloxKeys& keys, uint32_t tensor, uint32_t tag, uint64_t first_block, int64_t n_blocks,

@@ -1,0 +1,508 @@
+// Blackwell-native sweep for 16-bit weights with a rank > 8 subspace:
+//     theta <- rnd(theta + c (a Z + b U G))            (Eq. (perturbation) applied as in Algorithm 1)
+//
+// The generator and the Gaussian transform alone fill about 80 % of an SM's issue slots at the rate
+// HBM can feed the weights, so everything else is taken out of the SM's instruction stream:
+//
+//   * TMA brings a 128-row x NS-column tile of theta (and the matching 128 x KP tiles of U, pre-split
+//     into bf16 hi/lo) into shared memory, and writes the finished tile back; no thread issues a
+//     global load or store for the weights.
+//   * tcgen05.mma builds   D = theta + c b U G   in tensor memory (fp32):
+//       - "theta" enters through identity products  D[:, 16j:16j+16] = theta[:, 16j:16j+16] * I16
+//         with theta's own 16-bit tile as the A operand, which unpacks it to fp32 exactly, for free;
+//       - U G is accumulated on top as  Ulo Ghi + Uhi Glo + Uhi Ghi  (bf16 split operands,
+//         about 2^-16 relative error per term), the strip of c b G living in shared memory as the
+//         K-major B operand for all row tiles of a work item.
+//   * The sixteen epilogue warps read D with tcgen05.ld (one row per thread), add the isotropic
+//     normals (Philox4x32-10 + Box-Muller in registers), round to the storage type and write the
+//     tile into the shared-memory buffer the TMA store reads.
+//
+// Warp roles: warp 0 = TMA producer (loads and stores), warp 1 = MMA issuer and owner of the tensor
+// memory allocation, warps 2..17 = epilogue.  One CTA per SM (the shared-memory footprint
+// enforces it), persistent over a static round-robin list of work items.
+//
+// Every wait on an mbarrier is bounded: when a wait gives up it records where in *p.error, raises a
+// CTA-wide abort flag, and all roles fall through to the common exit, where the producer drains its
+// outstanding copies and warp 1 returns the tensor memory.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "zgr_device.cuh"
+#include "zgr_kernels.h"
+
+namespace zgr {
+namespace {
+
+constexpr int kEpiWarps = 16;
+constexpr int kUmmaThreads = 32 * (2 + kEpiWarps);
+constexpr unsigned long long kWaitLimitCycles = 4000000000ull;  // ~2 s at 2 GHz
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if it gave up or the CTA is already aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* error, int where) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      *abort_flag = 1;
+      atomicCAS(error, 0, where);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+               "l"(tmap), "r"(bar), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const void* tmap, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tmap), "r"(src), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,"
+      "%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]),
+        "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
+        "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]),
+        "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major operand whose rows are `row_bytes` (32, 64 or 128)
+// long and swizzled with the matching mode: eight rows form one swizzle atom, atoms follow each
+// other every 8*row_bytes (the stride byte offset); the leading byte offset is not used by
+// swizzled K-major layouts and is set to 1 (16 bytes).  Bits 46-47 = 1: Blackwell descriptor.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, int row_bytes) {
+  const uint64_t layout = row_bytes == 128 ? 2ull : (row_bytes == 64 ? 4ull : 6ull);
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFF);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(((8 * row_bytes) >> 4) & 0x3FFF) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= layout << 61;
+  return d;
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, A and B both `fmt` (0 = f16, 1 = bf16), both
+// K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t make_idesc(int fmt, int n) {
+  return (1u << 4) | (static_cast<uint32_t>(fmt) << 7) | (static_cast<uint32_t>(fmt) << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(128 >> 4) << 24);
+}
+// XOR swizzle of a byte offset inside a buffer aligned to 1024 bytes (rows of row_bytes bytes).
+__device__ __forceinline__ uint32_t swizzle(uint32_t off, int row_bytes) {
+  const uint32_t mask = row_bytes == 128 ? 7u : (row_bytes == 64 ? 3u : 1u);
+  return off ^ (((off >> 7) & mask) << 4);
+}
+
+template <typename T>
+struct Pack16;
+template <>
+struct Pack16<__nv_bfloat16> {
+  static constexpr int kFmt = 1;
+  static constexpr uint16_t kOne = 0x3F80;
+  static __device__ __forceinline__ uint32_t pack(float a, float b) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&h);
+  }
+};
+template <>
+struct Pack16<__half> {
+  static constexpr int kFmt = 0;
+  static constexpr uint16_t kOne = 0x3C00;
+  static __device__ __forceinline__ uint32_t pack(float a, float b) {
+    const __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&h);
+  }
+};
+
+__device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __uint_as_float(hi << 16), x1 - __uint_as_float(hi & 0xFFFF0000u));
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+template <int KP>
+struct UmmaCfg {
+  static constexpr int NS = KP == 64 ? 128 : 256;          // columns per strip / per accumulator buffer
+  static constexpr int STAGES = KP == 64 ? 3 : 2;
+  static constexpr int ROWB = KP * 2;                      // bytes per row of the U and G operands
+  static constexpr int THETA_BYTES = 128 * NS * 2;         // NS/64 boxes of 128 rows x 128 B
+  static constexpr int U_BYTES = 128 * ROWB;               // one of hi / lo
+  static constexpr int STAGE_BYTES = THETA_BYTES + 2 * U_BYTES;
+  static constexpr int G_BYTES = NS * ROWB;                // one of hi / lo
+  static constexpr int ID_BYTES = 1024;                    // 16 x 16 identity (512 B), padded to the swizzle alignment
+  static constexpr int BAR_BYTES = 1024;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * G_BYTES + ID_BYTES + BAR_BYTES + 1024 /* alignment slack */;
+  static constexpr int TMEM_COLS = 2 * NS;
+  static constexpr int COLS_PER_WARP = NS / (kEpiWarps / 4);
+};
+
+struct TileCoord {
+  int32_t tensor;
+  int32_t col0;
+  int32_t row0;
+  int32_t ncols;
+};
+
+}  // namespace
+
+template <typename T, int BITS, int KP>
+__global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
+                                                                     int* __restrict__ error) {
+  using Cfg = UmmaCfg<KP>;
+  constexpr int NS = Cfg::NS, S = Cfg::STAGES, ROWB = Cfg::ROWB;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint8_t* stage_base = smem;
+  uint8_t* g_hi = smem + S * Cfg::STAGE_BYTES;
+  uint8_t* g_lo = g_hi + Cfg::G_BYTES;
+  uint8_t* ident = g_lo + Cfg::G_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ident + Cfg::ID_BYTES);
+  // barrier indices
+  const uint32_t bar0 = smem_u32(bars);
+  auto BAR_FULL = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(s); };
+  auto BAR_OUT = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(S + s); };
+  auto BAR_ACC_FULL = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + b); };
+  auto BAR_ACC_EMPTY = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + 2 + b); };
+  const uint32_t BAR_G = bar0 + 8u * static_cast<uint32_t>(2 * S + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 5);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(BAR_FULL(s), 1);
+      mbar_init(BAR_OUT(s), kEpiWarps);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(BAR_ACC_FULL(b), 1);
+      mbar_init(BAR_ACC_EMPTY(b), kEpiWarps);
+    }
+    mbar_init(BAR_G, kEpiWarps);
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  // 16 x 16 identity in the storage type, K-major rows of 32 bytes, 32-byte swizzle
+  for (int i = threadIdx.x; i < 256; i += kUmmaThreads) {
+    const int n = i >> 4, k = i & 15;
+    *reinterpret_cast<uint16_t*>(ident + swizzle(static_cast<uint32_t>(n * 32 + k * 2), 32)) = (n == k) ? Pack16<T>::kOne : uint16_t(0);
+  }
+  fence_proxy_async();
+  __syncthreads();
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), Cfg::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // The three roles walk the same sequence of (item, row tile) pairs.
+  if (warp == 0) {
+    // ===================================== TMA producer =====================================
+    if (lane == 0) {
+      TileCoord ring[S];
+      int t = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x) {
+        const WorkItem w = p.items[it];
+        const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
+        for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
+          const int s = t % S;
+          if (t >= S) {
+            // the epilogue has written tile t-S into this stage: store it, then the stage is free
+            if (!mbar_wait(BAR_OUT(s), ((t / S) - 1) & 1, abort_flag, error, 1)) { ok = false; break; }
+            const TileCoord& o = ring[s];
+            const CUtensorMap* tm = tmaps + 3 * o.tensor;
+            const uint32_t src = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
+            for (int c = 0; c * 64 < o.ncols; ++c) tma_store_2d(tm, o.col0 + 64 * c, o.row0, src + c * 16384);
+            tma_commit();
+            tma_wait_read0();
+          }
+          ring[s] = TileCoord{w.tensor, static_cast<int32_t>(w.col0), row0, w.ncols};
+          const CUtensorMap* tm = tmaps + 3 * w.tensor;
+          const int nbox = (w.ncols + 63) / 64;
+          const uint32_t dst = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
+          mbar_arrive_expect_tx(BAR_FULL(s), static_cast<uint32_t>(nbox * 16384 + 2 * Cfg::U_BYTES));
+          for (int c = 0; c < nbox; ++c) tma_load_2d(dst + c * 16384, tm, static_cast<int>(w.col0) + 64 * c, row0, BAR_FULL(s));
+          tma_load_2d(dst + Cfg::THETA_BYTES, tm + 1, 0, row0, BAR_FULL(s));
+          tma_load_2d(dst + Cfg::THETA_BYTES + Cfg::U_BYTES, tm + 2, 0, row0, BAR_FULL(s));
+        }
+      }
+      // drain: store the last tiles
+      const int total = t;
+      for (int u = (total > S ? total - S : 0); u < total && ok; ++u) {
+        const int s = u % S;
+        if (!mbar_wait(BAR_OUT(s), (u / S) & 1, abort_flag, error, 2)) { ok = false; break; }
+        const TileCoord& o = ring[s];
+        const CUtensorMap* tm = tmaps + 3 * o.tensor;
+        const uint32_t src = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
+        for (int c = 0; c * 64 < o.ncols; ++c) tma_store_2d(tm, o.col0 + 64 * c, o.row0, src + c * 16384);
+        tma_commit();
+      }
+      if (!ok) {
+        // aborting: let the loads already issued land before the CTA gives up its shared memory
+        for (int u = (total > S ? total - S : 0); u < total; ++u) {
+          const unsigned long long t0 = clock64();
+          while (!mbar_try_wait(BAR_FULL(u % S), (u / S) & 1) && clock64() - t0 < kWaitLimitCycles) {
+          }
+        }
+      }
+      tma_wait_all0();
+    }
+  } else if (warp == 1) {
+    // ===================================== MMA issuer =====================================
+    if (lane == 0) {
+      const uint32_t idesc_id = make_idesc(Pack16<T>::kFmt, 16);
+      const uint32_t idesc_ug = make_idesc(1, NS);
+      const uint64_t desc_id = make_desc(smem_u32(ident), 32);
+      const uint64_t desc_ghi = make_desc(smem_u32(g_hi), ROWB);
+      const uint64_t desc_glo = make_desc(smem_u32(g_lo), ROWB);
+      int t = 0, item_no = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x, ++item_no) {
+        const WorkItem w = p.items[it];
+        if (!mbar_wait(BAR_G, item_no & 1, abort_flag, error, 3)) break;
+        tc_fence_after();
+        const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
+        const int nbox = (w.ncols + 63) / 64;
+        for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
+          const int s = t % S, b = t & 1;
+          if (!mbar_wait(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
+          if (t >= 2 && !mbar_wait(BAR_ACC_EMPTY(b), ((t >> 1) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sbase = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
+          const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
+          // theta -> fp32, 16 columns at a time
+          for (int c = 0; c < nbox; ++c)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma(d + static_cast<uint32_t>(64 * c + 16 * k), make_desc(sbase + c * 16384 + 32 * k, 128), desc_id, idesc_id, 0u);
+          // + c b U G, split operands
+          const uint32_t uhi = sbase + Cfg::THETA_BYTES, ulo = uhi + Cfg::U_BYTES;
+#pragma unroll
+          for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(ulo + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+#pragma unroll
+          for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_glo + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+#pragma unroll
+          for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+          umma_commit(BAR_ACC_FULL(b));
+        }
+      }
+    }
+  } else {
+    // ===================================== epilogue warps =====================================
+    const int e = warp - 2;                 // 0..15
+    const int quad = warp & 3;              // tensor-memory lane quadrant this warp may read
+    const int cgrp = e >> 2;                // which group of COLS_PER_WARP columns
+    const int et = e * 32 + lane;           // 0..511
+    constexpr int CPW = Cfg::COLS_PER_WARP;
+    int t = 0, item_no = 0;
+    bool ok = true;
+    for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x, ++item_no) {
+      const WorkItem w = p.items[it];
+      const TensorDesc& td = p.tensors[w.tensor];
+      const uint32_t tid = static_cast<uint32_t>(td.id);
+      const int r = td.rank;
+      // ---- coefficient strip c b G -> K-major hi/lo operands (all MMAs of the previous item are
+      //      complete: this warp has waited for the accumulator of its last tile) ----
+      for (int idx = et; idx < (KP / 2) * (NS / 8); idx += kEpiWarps * 32) {
+        const int kp = idx / (NS / 8), o = idx % (NS / 8);
+        const int cc = 8 * o;
+        float g0[8], g1[8];
+        if (cc < w.ncols && 2 * kp < r) {
+          coeffs8<BITS, false>(td, p.keys, p.unit, p.cb, 2 * kp, w.col0 + cc, g0);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) g0[i] = 0.0f;
+        }
+        if (cc < w.ncols && 2 * kp + 1 < r) {
+          coeffs8<BITS, false>(td, p.keys, p.unit, p.cb, 2 * kp + 1, w.col0 + cc, g1);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) g1[i] = 0.0f;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          uint32_t hi, lo;
+          split_bf16(g0[i], g1[i], hi, lo);
+          const uint32_t off = swizzle(static_cast<uint32_t>((cc + i) * ROWB + 4 * kp), ROWB);
+          *reinterpret_cast<uint32_t*>(g_hi + off) = hi;
+          *reinterpret_cast<uint32_t*>(g_lo + off) = lo;
+        }
+      }
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR_G);
+
+      const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
+      const bool active = cgrp * CPW < w.ncols;
+      for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
+        const int s = t % S, b = t & 1;
+        if (!mbar_wait(BAR_ACC_FULL(b), (t >> 1) & 1, abort_flag, error, 6)) { ok = false; break; }
+        tc_fence_after();
+        if (active) {
+          const int row_in_tile = 32 * quad + lane;
+          const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
+          uint8_t* out_tile = stage_base + s * Cfg::STAGE_BYTES;
+          // Philox block index of this thread's first octet (16-bit mode: one block per octet)
+          const uint64_t e_first = static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + cgrp * CPW);
+#pragma unroll 1
+          for (int g32 = 0; g32 < CPW / 32; ++g32) {
+            const int col_local = cgrp * CPW + 32 * g32;      // within the strip
+            uint32_t v[32];
+            tmem_ld32(tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(b * NS + col_local), v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int o = 0; o < 4; ++o) {
+              float z[8];
+              normals8<BITS, false>(p.keys, tid, 0u, e_first + static_cast<uint64_t>(32 * g32 + 8 * o), p.iso, z);
+              uint32_t q[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                q[i] = Pack16<T>::pack(__uint_as_float(v[8 * o + 2 * i]) + z[2 * i], __uint_as_float(v[8 * o + 2 * i + 1]) + z[2 * i + 1]);
+              const int col = col_local + 8 * o;              // column within the strip
+              const uint32_t off = static_cast<uint32_t>((col >> 6) * 16384 + row_in_tile * 128 + (col & 63) * 2);
+              *reinterpret_cast<uint4*>(out_tile + swizzle(off, 128)) = make_uint4(q[0], q[1], q[2], q[3]);
+            }
+          }
+        }
+        tc_fence_before();
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(BAR_ACC_EMPTY(b));
+          mbar_arrive(BAR_OUT(s));
+        }
+      }
+    }
+  }
+
+  // ---- common exit ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+}
+
+// U (rows x r fp32) -> two row-major bf16 matrices (hi, lo), rows padded to a multiple of 128 and
+// columns to KP with zeros: the TMA source of the A operand.
+__global__ void split_subspace_rowmajor_kernel(const float* __restrict__ U, int64_t rows, int r, int kp, int64_t rows_pad,
+                                               __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+  if (idx >= rows_pad * kp) return;
+  const int64_t row = idx / kp;
+  const int k = static_cast<int>(idx % kp);
+  const float x = (row < rows && k < r) ? U[row * r + k] : 0.0f;
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  hi[idx] = h;
+  lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+size_t umma_smem_bytes(int kpad) {
+  return kpad == 16 ? UmmaCfg<16>::SMEM_BYTES : (kpad == 32 ? UmmaCfg<32>::SMEM_BYTES : UmmaCfg<64>::SMEM_BYTES);
+}
+int umma_strip_cols(int kpad) { return kpad == 64 ? 128 : 256; }
+
+namespace {
+template <typename T, int BITS>
+cudaError_t launch_umma_kp(int kpad, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
+#define ZGR_LAUNCH_UMMA(KPV)                                                                                       \
+  {                                                                                                                \
+    auto k = sweep_umma_kernel<T, BITS, KPV>;                                                                      \
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<KPV>::SMEM_BYTES); \
+    if (e != cudaSuccess) return e;                                                                                \
+    k<<<grid, kUmmaThreads, UmmaCfg<KPV>::SMEM_BYTES, st>>>(p, tmaps, error);                                      \
+  }
+  if (kpad == 16) ZGR_LAUNCH_UMMA(16)
+  else if (kpad == 32) ZGR_LAUNCH_UMMA(32)
+  else ZGR_LAUNCH_UMMA(64)
+#undef ZGR_LAUNCH_UMMA
+  return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
+  if (kc.dtype == 2) {
+    return kc.bits == 32 ? launch_umma_kp<__nv_bfloat16, 32>(kc.kpad, p, tmaps, error, grid, st)
+                         : launch_umma_kp<__nv_bfloat16, 16>(kc.kpad, p, tmaps, error, grid, st);
+  }
+  if (kc.dtype == 1) {
+    return kc.bits == 32 ? launch_umma_kp<__half, 32>(kc.kpad, p, tmaps, error, grid, st) : launch_umma_kp<__half, 16>(kc.kpad, p, tmaps, error, grid, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st) {
+  const int64_t n = rows_pad * kp;
+  const int block = 256;
+  split_subspace_rowmajor_kernel<<<static_cast<unsigned>((n + block - 1) / block), block, 0, st>>>(
+      U, rows, r, kp, rows_pad, static_cast<__nv_bfloat16*>(hi), static_cast<__nv_bfloat16*>(lo));
+  return cudaGetLastError();
+}
+
+}  // namespace zgr

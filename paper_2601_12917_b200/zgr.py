@@ -36,7 +36,7 @@ class ZgrKernelTime(ctypes.Structure):
                 ("elements", ctypes.c_int64), ("ms_total", ctypes.c_double)]
 
 
-PATH_NAMES = {0: "iso", 1: "fma", 2: "mma", 3: "generic"}
+PATH_NAMES = {0: "iso", 1: "fma", 2: "mma", 3: "generic", 4: "umma"}
 
 
 class ZgrError(RuntimeError):
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.zgr_profile_read.argtypes = [vp, ctypes.POINTER(ZgrKernelTime), i32, ctypes.POINTER(i32)]
         L.zgr_tensor_norms_noalloc.argtypes = [vp, u64, i32, vp, vp]
         L.zgr_tensor_norms_noalloc.restype = ctypes.c_int
+        L.zgr_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+        L.zgr_device_status.restype = ctypes.c_int
         L.zgr_launch_count.argtypes = [vp]
         L.zgr_launch_count.restype = i64
         L.zgr_destroy.argtypes = [vp]
@@ -197,6 +199,12 @@ class Zgr:
         out = torch.empty(w.shape, dtype=torch.float32, device=w.device)
         _check(lib().zgr_debug_z(self._h, seed, tensor, out.data_ptr(), _stream_ptr(stream)), "zgr_debug_z")
         return out
+
+    def device_status(self) -> int:
+        """Synchronise and return the device-side status code (0 = healthy)."""
+        code = ctypes.c_int32()
+        _check(lib().zgr_device_status(self._h, ctypes.byref(code)), "zgr_device_status")
+        return code.value
 
     def scalars(self):
         a, b = ctypes.c_double(), ctypes.c_double()

@@ -112,6 +112,7 @@ class Pair:
         before = [oracle.decode(t.theta, t.dtype) for t in ots]
         fn()
         torch.cuda.synchronize()
+        assert self.lib.device_status() == 0, "a kernel abandoned a bounded wait"
         reports, exps = [], []
         for l, t in enumerate(ots):
             oracle.sweep_tensor(t, seed, l, self.bits, self.a, self.b, c)
