@@ -56,10 +56,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(2000u) /* suspend-time hint in ns: waiting warps sleep instead of spinning */
       : "memory");
   return ok != 0;
 }
@@ -183,8 +183,9 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 
 template <int KP>
 struct UmmaCfg {
-  static constexpr int NS = KP == 64 ? 128 : 256;          // columns per strip / per accumulator buffer
-  static constexpr int STAGES = KP == 64 ? 3 : 2;
+  static constexpr int NS = 128;                           // columns per strip / per accumulator buffer
+  static constexpr int STAGES = KP == 64 ? 3 : (KP == 32 ? 4 : 5);
+  static constexpr int NACC = 4;                           // accumulator buffers in tensor memory
   static constexpr int ROWB = KP * 2;                      // bytes per row of the U and G operands
   static constexpr int THETA_BYTES = 128 * NS * 2;         // NS/64 boxes of 128 rows x 128 B
   static constexpr int U_BYTES = 128 * ROWB;               // one of hi / lo
@@ -193,7 +194,7 @@ struct UmmaCfg {
   static constexpr int ID_BYTES = 1024;                    // 16 x 16 identity (512 B), padded to the swizzle alignment
   static constexpr int BAR_BYTES = 1024;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * G_BYTES + ID_BYTES + BAR_BYTES + 1024 /* alignment slack */;
-  static constexpr int TMEM_COLS = 2 * NS;
+  static constexpr int TMEM_COLS = NACC * NS;
   static constexpr int COLS_PER_WARP = NS / (kEpiWarps / 4);
 };
 
@@ -210,7 +211,7 @@ template <typename T, int BITS, int KP>
 __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
                                                                      int* __restrict__ error) {
   using Cfg = UmmaCfg<KP>;
-  constexpr int NS = Cfg::NS, S = Cfg::STAGES, ROWB = Cfg::ROWB;
+  constexpr int NS = Cfg::NS, S = Cfg::STAGES, ROWB = Cfg::ROWB, NACC = Cfg::NACC;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   uint8_t* stage_base = smem;
@@ -223,9 +224,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
   auto BAR_FULL = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(s); };
   auto BAR_OUT = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(S + s); };
   auto BAR_ACC_FULL = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + b); };
-  auto BAR_ACC_EMPTY = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + 2 + b); };
-  const uint32_t BAR_G = bar0 + 8u * static_cast<uint32_t>(2 * S + 4);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 5);
+  auto BAR_ACC_EMPTY = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + NACC + b); };
+  const uint32_t BAR_G = bar0 + 8u * static_cast<uint32_t>(2 * S + 2 * NACC);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2 * NACC + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -235,7 +236,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       mbar_init(BAR_FULL(s), 1);
       mbar_init(BAR_OUT(s), kEpiWarps);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < NACC; ++b) {
       mbar_init(BAR_ACC_FULL(b), 1);
       mbar_init(BAR_ACC_EMPTY(b), kEpiWarps);
     }
@@ -329,9 +330,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
         const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
         const int nbox = (w.ncols + 63) / 64;
         for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
-          const int s = t % S, b = t & 1;
+          const int s = t % S, b = t % NACC;
           if (!mbar_wait(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
-          if (t >= 2 && !mbar_wait(BAR_ACC_EMPTY(b), ((t >> 1) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
+          if (t >= NACC && !mbar_wait(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sbase = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
           const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
@@ -400,8 +401,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
       const bool active = cgrp * CPW < w.ncols;
       for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
-        const int s = t % S, b = t & 1;
-        if (!mbar_wait(BAR_ACC_FULL(b), (t >> 1) & 1, abort_flag, error, 6)) { ok = false; break; }
+        const int s = t % S, b = t % NACC;
+        if (!mbar_wait(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
         tc_fence_after();
         if (active) {
           const int row_in_tile = 32 * quad + lane;
@@ -466,7 +467,7 @@ __global__ void split_subspace_rowmajor_kernel(const float* __restrict__ U, int6
 size_t umma_smem_bytes(int kpad) {
   return kpad == 16 ? UmmaCfg<16>::SMEM_BYTES : (kpad == 32 ? UmmaCfg<32>::SMEM_BYTES : UmmaCfg<64>::SMEM_BYTES);
 }
-int umma_strip_cols(int kpad) { return kpad == 64 ? 128 : 256; }
+int umma_strip_cols(int kpad) { (void)kpad; return 128; }
 
 namespace {
 template <typename T, int BITS>
