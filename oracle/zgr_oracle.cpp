@@ -88,24 +88,26 @@ inline double box_muller(double u1, double u2, int which) {
 
 // Standard normal attached to element index e of stream (seed, tensor, tag)  [z ~ N(0, I_d), Eq. (ZOO)].
 //   bits == 32: block j = e/4 serves elements 4j..4j+3; words (x0,x1) -> normals 0,1 and (x2,x3) ->
-//               normals 2,3; u1 = odd_uniform(x_even >> 9, 23), u2 = odd_uniform(x_odd >> 9, 23).
+//               normals 2,3; the uniform field of a word is its low 23 bits: k = x & 0x7FFFFF.
 //   bits == 16: block j = e/8 serves elements 8j..8j+7; word x_w -> normals 2w, 2w+1 with
-//               u1 from its high 16 bits and u2 from its low 16 bits.
+//               k1 = bits 7..22 of x (radius) and k2 = bits 7..22 of x rotated by 16, i.e. the
+//               remaining bits 23..31 (low part of k2) and 0..6 (high part of k2) (angle).
 double normal_at(uint64_t seed, uint32_t tensor, uint32_t tag, int bits, uint64_t e) {
   uint32_t x[4];
   if (bits == 32) {
     stream_block(seed, e / 4, tensor, tag, x);
     const int w = static_cast<int>(e % 4);
     const int pair = w / 2;
-    const double u1 = odd_uniform(x[2 * pair] >> 9, 23);
-    const double u2 = odd_uniform(x[2 * pair + 1] >> 9, 23);
+    const double u1 = odd_uniform(x[2 * pair] & 0x7FFFFFu, 23);
+    const double u2 = odd_uniform(x[2 * pair + 1] & 0x7FFFFFu, 23);
     return box_muller(u1, u2, w % 2);
   }
   stream_block(seed, e / 8, tensor, tag, x);
   const int w = static_cast<int>(e % 8);
   const uint32_t word = x[w / 2];
-  const double u1 = odd_uniform(word >> 16, 16);
-  const double u2 = odd_uniform(word & 0xFFFFu, 16);
+  const uint32_t rot = (word << 16) | (word >> 16);
+  const double u1 = odd_uniform((word >> 7) & 0xFFFFu, 16);
+  const double u2 = odd_uniform((rot >> 7) & 0xFFFFu, 16);
   return box_muller(u1, u2, w % 2);
 }
 

@@ -93,10 +93,17 @@ __device__ __forceinline__ void box_muller(uint32_t m1, uint32_t m2, const Norma
   }
 }
 
+// Mantissa-position uniform fields of a generator word (see box_muller): one logic operation each.
+//   32-bit mode: the low 23 bits of the word.
+//   16-bit mode: bits 7..22 of the word (radius) and bits 7..22 of the word rotated by 16 (angle).
+__device__ __forceinline__ uint32_t field23(uint32_t x) { return x & 0x7FFFFFu; }
+__device__ __forceinline__ uint32_t field16a(uint32_t x) { return x & 0x7FFF80u; }
+__device__ __forceinline__ uint32_t field16b(uint32_t x) { return __funnelshift_l(x, x, 16) & 0x7FFF80u; }
+
 // Eight consecutive normals of stream (tensor, tag) starting at element e (a multiple of 8), each
 // already multiplied by the scale folded into `ns`.
 //   BITS == 32: blocks e/4 and e/4+1; words (x0,x1) -> normals 0,1 and (x2,x3) -> normals 2,3.
-//   BITS == 16: block e/8; word w -> normals 2w, 2w+1 from its high and low 16 bits.
+//   BITS == 16: block e/8; word w -> normals 2w, 2w+1.
 template <int BITS, bool PRECISE>
 __device__ __forceinline__ void normals8(const PhiloxKeys& keys, uint32_t tensor, uint32_t tag, uint64_t e, const NormalScale& ns,
                                          float (&z)[8]) {
@@ -105,14 +112,44 @@ __device__ __forceinline__ void normals8(const PhiloxKeys& keys, uint32_t tensor
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       philox_block((e >> 2) + h, tensor, tag, keys, x);
-      box_muller<PRECISE>(x[0] >> 9, x[1] >> 9, ns, z[4 * h + 0], z[4 * h + 1]);
-      box_muller<PRECISE>(x[2] >> 9, x[3] >> 9, ns, z[4 * h + 2], z[4 * h + 3]);
+      box_muller<PRECISE>(field23(x[0]), field23(x[1]), ns, z[4 * h + 0], z[4 * h + 1]);
+      box_muller<PRECISE>(field23(x[2]), field23(x[3]), ns, z[4 * h + 2], z[4 * h + 3]);
     }
   } else {
     philox_block(e >> 3, tensor, tag, keys, x);
 #pragma unroll
-    for (int w = 0; w < 4; ++w)
-      box_muller<PRECISE>((x[w] >> 9) & 0x7FFF80u, (x[w] << 7) & 0x7FFF80u, ns, z[2 * w], z[2 * w + 1]);
+    for (int w = 0; w < 4; ++w) box_muller<PRECISE>(field16a(x[w]), field16b(x[w]), ns, z[2 * w], z[2 * w + 1]);
+  }
+}
+
+// Fast transform fused with its consumer: acc0 += s rho cos(phi), acc1 += s rho sin(phi).
+__device__ __forceinline__ void box_muller_acc(uint32_t m1, uint32_t m2, const NormalScale& ns, float& acc0, float& acc1) {
+  const float u1 = __uint_as_float(0x3F800000u | m1) + ns.u1_off;
+  const float t2 = __uint_as_float(0x3F800000u | m2);
+  const float rho = sqrt_approx(fabsf(ns.kr * lg2_approx(u1)));
+  const float phi = fmaf(t2, 6.28318530717958647692f, ns.phase);
+  acc0 = fmaf(rho, cos_approx(phi), acc0);
+  acc1 = fmaf(rho, sin_approx(phi), acc1);
+}
+
+// acc[0..7] += the eight scaled normals of octet number `oct` (= element index / 8, as two 32-bit
+// halves) of stream (tensor, tag 0).  Hardware-approximation transform only.
+template <int BITS>
+__device__ __forceinline__ void normals8_acc(const PhiloxKeys& keys, uint32_t tensor, uint32_t oct_lo, uint32_t oct_hi, const NormalScale& ns,
+                                             float (&acc)[8]) {
+  uint32_t x[4];
+  if (BITS == 32) {
+    const uint32_t b_lo = oct_lo << 1, b_hi = (oct_hi << 1) | (oct_lo >> 31);   // block 2*oct; 2*oct + 1 cannot carry
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      philox4x32_10(b_lo + h, b_hi, tensor, 0u, keys, x);
+      box_muller_acc(field23(x[0]), field23(x[1]), ns, acc[4 * h + 0], acc[4 * h + 1]);
+      box_muller_acc(field23(x[2]), field23(x[3]), ns, acc[4 * h + 2], acc[4 * h + 3]);
+    }
+  } else {
+    philox4x32_10(oct_lo, oct_hi, tensor, 0u, keys, x);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) box_muller_acc(field16a(x[w]), field16b(x[w]), ns, acc[2 * w], acc[2 * w + 1]);
   }
 }
 
@@ -124,12 +161,12 @@ __device__ __forceinline__ float normal1(const PhiloxKeys& keys, uint32_t tensor
   if (BITS == 32) {
     philox_block(e >> 2, tensor, tag, keys, x);
     const int pair = static_cast<int>(e & 3) >> 1;
-    box_muller<PRECISE>((pair ? x[2] : x[0]) >> 9, (pair ? x[3] : x[1]) >> 9, ns, n0, n1);
+    box_muller<PRECISE>(field23(pair ? x[2] : x[0]), field23(pair ? x[3] : x[1]), ns, n0, n1);
   } else {
     philox_block(e >> 3, tensor, tag, keys, x);
     const int w = static_cast<int>(e & 7) >> 1;
     const uint32_t word = w == 0 ? x[0] : (w == 1 ? x[1] : (w == 2 ? x[2] : x[3]));
-    box_muller<PRECISE>((word >> 9) & 0x7FFF80u, (word << 7) & 0x7FFF80u, ns, n0, n1);
+    box_muller<PRECISE>(field16a(word), field16b(word), ns, n0, n1);
   }
   return (e & 1) ? n1 : n0;
 }

@@ -63,17 +63,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if it gave up or the CTA is already aborting.
+// Bounded wait.  Returns false if it gave up or the CTA is already aborting.  The abort flag and
+// the clock are looked at only every 256 polls, so a waiting warp costs few issue slots;
+// BACKOFF adds a short sleep between polls for the two single-thread roles, which run ahead of the
+// epilogue and must not steal issue slots from the warps that share their scheduler.
+template <bool BACKOFF>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* error, int where) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = clock64();
+  uint32_t polls = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
-      atomicCAS(error, 0, where);
-      return false;
+    if (BACKOFF) __nanosleep(64);
+    if ((++polls & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        atomicCAS(error, 0, where);
+        return false;
+      }
     }
   }
 }
@@ -114,16 +122,12 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t b
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,"
-      "%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]),
-        "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
-        "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]),
-        "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]),
+                 "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+               : "r"(taddr)
+               : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
           const int s = t % S;
           if (t >= S) {
             // the epilogue has written tile t-S into this stage: store it, then the stage is free
-            if (!mbar_wait(BAR_OUT(s), ((t / S) - 1) & 1, abort_flag, error, 1)) { ok = false; break; }
+            if (!mbar_wait<true>(BAR_OUT(s), ((t / S) - 1) & 1, abort_flag, error, 1)) { ok = false; break; }
             const TileCoord& o = ring[s];
             const CUtensorMap* tm = tmaps + 3 * o.tensor;
             const uint32_t src = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
@@ -296,7 +300,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       const int total = t;
       for (int u = (total > S ? total - S : 0); u < total && ok; ++u) {
         const int s = u % S;
-        if (!mbar_wait(BAR_OUT(s), (u / S) & 1, abort_flag, error, 2)) { ok = false; break; }
+        if (!mbar_wait<true>(BAR_OUT(s), (u / S) & 1, abort_flag, error, 2)) { ok = false; break; }
         const TileCoord& o = ring[s];
         const CUtensorMap* tm = tmaps + 3 * o.tensor;
         const uint32_t src = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
@@ -325,14 +329,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       bool ok = true;
       for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x, ++item_no) {
         const WorkItem w = p.items[it];
-        if (!mbar_wait(BAR_G, item_no & 1, abort_flag, error, 3)) break;
+        if (!mbar_wait<true>(BAR_G, item_no & 1, abort_flag, error, 3)) break;
         tc_fence_after();
         const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
         const int nbox = (w.ncols + 63) / 64;
         for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
           const int s = t % S, b = t % NACC;
-          if (!mbar_wait(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
-          if (t >= NACC && !mbar_wait(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
+          if (!mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
+          if (t >= NACC && !mbar_wait<true>(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sbase = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
           const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
@@ -400,34 +404,37 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
 
       const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
       const bool active = cgrp * CPW < w.ncols;
+      static_assert(CPW == 32, "the epilogue below handles 32 columns per warp");
+      const uint32_t tmem_warp = tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(cgrp * CPW);
       for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
         const int s = t % S, b = t % NACC;
-        if (!mbar_wait(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
+        if (!mbar_wait<false>(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
         tc_fence_after();
         if (active) {
           const int row_in_tile = 32 * quad + lane;
           const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
-          uint8_t* out_tile = stage_base + s * Cfg::STAGE_BYTES;
-          // Philox block index of this thread's first octet (16-bit mode: one block per octet)
-          const uint64_t e_first = static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + cgrp * CPW);
-#pragma unroll 1
-          for (int g32 = 0; g32 < CPW / 32; ++g32) {
-            const int col_local = cgrp * CPW + 32 * g32;      // within the strip
-            uint32_t v[32];
-            tmem_ld32(tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(b * NS + col_local), v);
-            tmem_ld_wait();
+          // number of this thread's first octet in the tensor (element index / 8)
+          const uint64_t oct0 = (static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + cgrp * CPW)) >> 3;
+          const uint32_t oct0_lo = static_cast<uint32_t>(oct0), oct0_hi = static_cast<uint32_t>(oct0 >> 32);
+          // output position: box (col / 64), row, 16-byte chunk XOR-swizzled with the row
+          uint8_t* out_box = stage_base + s * Cfg::STAGE_BYTES + ((cgrp * CPW) >> 6) * 16384 + row_in_tile * 128;
+          const uint32_t chunk0 = static_cast<uint32_t>(((cgrp * CPW) & 63) >> 3);
+          const uint32_t row_xor = static_cast<uint32_t>(row_in_tile & 7);
+          uint32_t h0[16], h1[16];
+          tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS), h0);
+          tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 16), h1);
+          tmem_ld_wait();
+          // four octets per thread, kept independent so that their generator chains interleave
 #pragma unroll
-            for (int o = 0; o < 4; ++o) {
-              float z[8];
-              normals8<BITS, false>(p.keys, tid, 0u, e_first + static_cast<uint64_t>(32 * g32 + 8 * o), p.iso, z);
-              uint32_t q[4];
+          for (int o = 0; o < 4; ++o) {
+            float acc[8];
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                q[i] = Pack16<T>::pack(__uint_as_float(v[8 * o + 2 * i]) + z[2 * i], __uint_as_float(v[8 * o + 2 * i + 1]) + z[2 * i + 1]);
-              const int col = col_local + 8 * o;              // column within the strip
-              const uint32_t off = static_cast<uint32_t>((col >> 6) * 16384 + row_in_tile * 128 + (col & 63) * 2);
-              *reinterpret_cast<uint4*>(out_tile + swizzle(off, 128)) = make_uint4(q[0], q[1], q[2], q[3]);
-            }
+            for (int i = 0; i < 8; ++i) acc[i] = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
+            const uint32_t lo = oct0_lo + static_cast<uint32_t>(o);
+            normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, acc);
+            const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
+                                       Pack16<T>::pack(acc[6], acc[7]));
+            *reinterpret_cast<uint4*>(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4)) = q;
           }
         }
         tc_fence_before();

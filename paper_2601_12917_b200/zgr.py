@@ -12,7 +12,7 @@ import os
 from typing import List, Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libzgr.so")
+LIB_PATH = os.environ.get("ZGR_LIBRARY", os.path.join(_HERE, "libzgr.so"))   # override: an alternative build of the same ABI
 
 OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5
 NOALLOC_MAX_TILES = 8192

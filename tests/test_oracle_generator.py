@@ -129,14 +129,17 @@ def _expected_normals_from_block(x, bits):
     out = []
     if bits == 32:
         for p in range(2):
-            u1 = (2 * (int(x[2 * p]) >> 9) + 1) / 2.0**24
-            u2 = (2 * (int(x[2 * p + 1]) >> 9) + 1) / 2.0**24
+            u1 = (2 * (int(x[2 * p]) & 0x7FFFFF) + 1) / 2.0**24
+            u2 = (2 * (int(x[2 * p + 1]) & 0x7FFFFF) + 1) / 2.0**24
             rho = math.sqrt(-2.0 * math.log(u1))
             out += [rho * math.cos(2 * math.pi * u2), rho * math.sin(2 * math.pi * u2)]
     else:
         for w in range(4):
-            u1 = (2 * (int(x[w]) >> 16) + 1) / 2.0**17
-            u2 = (2 * (int(x[w]) & 0xFFFF) + 1) / 2.0**17
+            xw = int(x[w])
+            k1 = (xw >> 7) & 0xFFFF                      # bits 7..22
+            k2 = (xw >> 23) | ((xw & 0x7F) << 9)         # bits 23..31 (low) and 0..6 (high)
+            u1 = (2 * k1 + 1) / 2.0**17
+            u2 = (2 * k2 + 1) / 2.0**17
             rho = math.sqrt(-2.0 * math.log(u1))
             out += [rho * math.cos(2 * math.pi * u2), rho * math.sin(2 * math.pi * u2)]
     return np.array(out)
