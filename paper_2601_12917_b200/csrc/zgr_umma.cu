@@ -86,6 +86,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+__device__ __forceinline__ void sts128(uint32_t saddr, const uint4& v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t saddr, uint32_t v) { asm volatile("st.shared.b32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory"); }
+
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -187,50 +192,56 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 
 template <int KP>
 struct UmmaCfg {
-  static constexpr int NS = 128;                           // columns per strip / per accumulator buffer
-  static constexpr int STAGES = KP == 64 ? 3 : (KP == 32 ? 4 : 5);
+  static constexpr int NS = 128;                           // columns per tile / per accumulator buffer
+  static constexpr int NSUB = KP == 64 ? 1 : (KP == 32 ? 2 : 4);   // adjacent tiles per row block that share one U tile
+  static constexpr int STAGES = KP == 64 ? 4 : 5;          // theta tiles in flight (loaded, transformed in place, stored)
+  static constexpr int USTAGES = 2;                        // U tiles in flight
   static constexpr int NACC = 4;                           // accumulator buffers in tensor memory
   static constexpr int ROWB = KP * 2;                      // bytes per row of the U and G operands
   static constexpr int THETA_BYTES = 128 * NS * 2;         // NS/64 boxes of 128 rows x 128 B
   static constexpr int U_BYTES = 128 * ROWB;               // one of hi / lo
-  static constexpr int STAGE_BYTES = THETA_BYTES + 2 * U_BYTES;
-  static constexpr int G_BYTES = NS * ROWB;                // one of hi / lo
+  static constexpr int G_BYTES = NS * ROWB;                // one of hi / lo, one tile's strip
   static constexpr int ID_BYTES = 1024;                    // 16 x 16 identity (512 B), padded to the swizzle alignment
   static constexpr int BAR_BYTES = 1024;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * G_BYTES + ID_BYTES + BAR_BYTES + 1024 /* alignment slack */;
+  static constexpr int SMEM_BYTES =
+      STAGES * THETA_BYTES + USTAGES * 2 * U_BYTES + NSUB * 2 * G_BYTES + ID_BYTES + BAR_BYTES + 1024 /* alignment slack */;
   static constexpr int TMEM_COLS = NACC * NS;
-  static constexpr int COLS_PER_WARP = NS / (kEpiWarps / 4);
+  static_assert(SMEM_BYTES <= 232448, "shared-memory budget of one CTA");
 };
 
 struct TileCoord {
   int32_t tensor;
   int32_t col0;
   int32_t row0;
-  int32_t ncols;
+  int32_t ncols;   // columns of this tile that exist in the tensor (<= 128)
 };
 
 }  // namespace
 
+// Work item = NSUB adjacent column tiles (a strip of up to 128*NSUB columns) x a range of rows.
+// Tiles are visited row block by row block, the NSUB tiles of a row block one after the other, so
+// that a CTA touches up to 256*NSUB contiguous bytes of every row and loads each U tile once.
 template <typename T, int BITS, int KP>
 __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
                                                                      int* __restrict__ error) {
   using Cfg = UmmaCfg<KP>;
-  constexpr int NS = Cfg::NS, S = Cfg::STAGES, ROWB = Cfg::ROWB, NACC = Cfg::NACC;
+  constexpr int NS = Cfg::NS, S = Cfg::STAGES, US = Cfg::USTAGES, ROWB = Cfg::ROWB, NACC = Cfg::NACC, NSUB = Cfg::NSUB;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  uint8_t* stage_base = smem;
-  uint8_t* g_hi = smem + S * Cfg::STAGE_BYTES;
-  uint8_t* g_lo = g_hi + Cfg::G_BYTES;
-  uint8_t* ident = g_lo + Cfg::G_BYTES;
+  uint8_t* theta_base = smem;                                           // S tiles
+  uint8_t* u_base = theta_base + S * Cfg::THETA_BYTES;                  // US x (hi, lo)
+  uint8_t* g_base = u_base + US * 2 * Cfg::U_BYTES;                     // NSUB x (hi, lo)
+  uint8_t* ident = g_base + NSUB * 2 * Cfg::G_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(ident + Cfg::ID_BYTES);
-  // barrier indices
   const uint32_t bar0 = smem_u32(bars);
-  auto BAR_FULL = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(s); };
-  auto BAR_OUT = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(S + s); };
-  auto BAR_ACC_FULL = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + b); };
-  auto BAR_ACC_EMPTY = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + NACC + b); };
-  const uint32_t BAR_G = bar0 + 8u * static_cast<uint32_t>(2 * S + 2 * NACC);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2 * NACC + 1);
+  auto BAR_FULL = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(s); };                          // theta tile landed
+  auto BAR_OUT = [&](int s) { return bar0 + 8u * static_cast<uint32_t>(S + s); };                       // result written into the stage
+  auto BAR_ACC_FULL = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + b); };              // accumulator complete
+  auto BAR_ACC_EMPTY = [&](int b) { return bar0 + 8u * static_cast<uint32_t>(2 * S + NACC + b); };      // accumulator read out
+  auto BAR_U_FULL = [&](int u) { return bar0 + 8u * static_cast<uint32_t>(2 * S + 2 * NACC + u); };     // U tile landed
+  auto BAR_U_FREE = [&](int u) { return bar0 + 8u * static_cast<uint32_t>(2 * S + 2 * NACC + US + u); };  // U tile consumed
+  const uint32_t BAR_G = bar0 + 8u * static_cast<uint32_t>(2 * S + 2 * NACC + 2 * US);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2 * NACC + 2 * US + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -238,11 +249,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(BAR_FULL(s), 1);
-      mbar_init(BAR_OUT(s), kEpiWarps);
+      mbar_init(BAR_OUT(s), kEpiWarps / 2);
     }
     for (int b = 0; b < NACC; ++b) {
       mbar_init(BAR_ACC_FULL(b), 1);
-      mbar_init(BAR_ACC_EMPTY(b), kEpiWarps);
+      mbar_init(BAR_ACC_EMPTY(b), kEpiWarps / 2);
+    }
+    for (int u = 0; u < US; ++u) {
+      mbar_init(BAR_U_FULL(u), 1);
+      mbar_init(BAR_U_FREE(u), 1);
     }
     mbar_init(BAR_G, kEpiWarps);
     *abort_flag = 0;
@@ -264,54 +279,67 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // The three roles walk the same sequence of (item, row tile) pairs.
+  // The three roles walk the same sequence of (item, row block, tile) triples; t counts tiles and
+  // rb counts row blocks over the whole life of the CTA, which fixes every ring slot and phase.
   if (warp == 0) {
     // ===================================== TMA producer =====================================
     if (lane == 0) {
       TileCoord ring[S];
-      int t = 0;
+      int t = 0, rb = 0;
       bool ok = true;
+      auto store_tile = [&](int s) {
+        const TileCoord& o = ring[s];
+        const CUtensorMap* tm = tmaps + 3 * o.tensor;
+        const uint32_t src = smem_u32(theta_base + s * Cfg::THETA_BYTES);
+        for (int c = 0; c * 64 < o.ncols; ++c) tma_store_2d(tm, o.col0 + 64 * c, o.row0, src + c * 16384);
+        tma_commit();
+      };
       for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x) {
         const WorkItem w = p.items[it];
+        const CUtensorMap* tm = tmaps + 3 * w.tensor;
         const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
-        for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
-          const int s = t % S;
-          if (t >= S) {
-            // the epilogue has written tile t-S into this stage: store it, then the stage is free
-            if (!mbar_wait<true>(BAR_OUT(s), ((t / S) - 1) & 1, abort_flag, error, 1)) { ok = false; break; }
-            const TileCoord& o = ring[s];
-            const CUtensorMap* tm = tmaps + 3 * o.tensor;
-            const uint32_t src = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
-            for (int c = 0; c * 64 < o.ncols; ++c) tma_store_2d(tm, o.col0 + 64 * c, o.row0, src + c * 16384);
-            tma_commit();
-            tma_wait_read0();
+        const int nsub = (w.ncols + NS - 1) / NS;
+        for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128, ++rb) {
+          const int u = rb % US;
+          if (rb >= US && !mbar_wait<true>(BAR_U_FREE(u), ((rb / US) - 1) & 1, abort_flag, error, 8)) { ok = false; break; }
+          const uint32_t udst = smem_u32(u_base + u * 2 * Cfg::U_BYTES);
+          mbar_arrive_expect_tx(BAR_U_FULL(u), static_cast<uint32_t>(2 * Cfg::U_BYTES));
+          tma_load_2d(udst, tm + 1, 0, row0, BAR_U_FULL(u));
+          tma_load_2d(udst + Cfg::U_BYTES, tm + 2, 0, row0, BAR_U_FULL(u));
+          for (int sub = 0; sub < nsub; ++sub, ++t) {
+            const int s = t % S;
+            if (t >= S) {
+              // the epilogue has written tile t-S into this stage: store it, then the stage is free
+              if (!mbar_wait<true>(BAR_OUT(s), ((t / S) - 1) & 1, abort_flag, error, 1)) { ok = false; break; }
+              store_tile(s);
+              tma_wait_read0();
+            }
+            const int col0 = static_cast<int>(w.col0) + NS * sub;
+            const int ncols = min(NS, w.ncols - NS * sub);
+            ring[s] = TileCoord{w.tensor, col0, row0, ncols};
+            const int nbox = (ncols + 63) / 64;
+            const uint32_t dst = smem_u32(theta_base + s * Cfg::THETA_BYTES);
+            mbar_arrive_expect_tx(BAR_FULL(s), static_cast<uint32_t>(nbox * 16384));
+            for (int c = 0; c < nbox; ++c) tma_load_2d(dst + c * 16384, tm, col0 + 64 * c, row0, BAR_FULL(s));
           }
-          ring[s] = TileCoord{w.tensor, static_cast<int32_t>(w.col0), row0, w.ncols};
-          const CUtensorMap* tm = tmaps + 3 * w.tensor;
-          const int nbox = (w.ncols + 63) / 64;
-          const uint32_t dst = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
-          mbar_arrive_expect_tx(BAR_FULL(s), static_cast<uint32_t>(nbox * 16384 + 2 * Cfg::U_BYTES));
-          for (int c = 0; c < nbox; ++c) tma_load_2d(dst + c * 16384, tm, static_cast<int>(w.col0) + 64 * c, row0, BAR_FULL(s));
-          tma_load_2d(dst + Cfg::THETA_BYTES, tm + 1, 0, row0, BAR_FULL(s));
-          tma_load_2d(dst + Cfg::THETA_BYTES + Cfg::U_BYTES, tm + 2, 0, row0, BAR_FULL(s));
         }
       }
       // drain: store the last tiles
       const int total = t;
-      for (int u = (total > S ? total - S : 0); u < total && ok; ++u) {
-        const int s = u % S;
-        if (!mbar_wait<true>(BAR_OUT(s), (u / S) & 1, abort_flag, error, 2)) { ok = false; break; }
-        const TileCoord& o = ring[s];
-        const CUtensorMap* tm = tmaps + 3 * o.tensor;
-        const uint32_t src = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
-        for (int c = 0; c * 64 < o.ncols; ++c) tma_store_2d(tm, o.col0 + 64 * c, o.row0, src + c * 16384);
-        tma_commit();
+      for (int v = (total > S ? total - S : 0); v < total && ok; ++v) {
+        if (!mbar_wait<true>(BAR_OUT(v % S), (v / S) & 1, abort_flag, error, 2)) { ok = false; break; }
+        store_tile(v % S);
       }
       if (!ok) {
         // aborting: let the loads already issued land before the CTA gives up its shared memory
-        for (int u = (total > S ? total - S : 0); u < total; ++u) {
+        for (int v = (total > S ? total - S : 0); v < total; ++v) {
           const unsigned long long t0 = clock64();
-          while (!mbar_try_wait(BAR_FULL(u % S), (u / S) & 1) && clock64() - t0 < kWaitLimitCycles) {
+          while (!mbar_try_wait(BAR_FULL(v % S), (v / S) & 1) && clock64() - t0 < kWaitLimitCycles) {
+          }
+        }
+        for (int v = (rb > US ? rb - US : 0); v < rb; ++v) {
+          const unsigned long long t0 = clock64();
+          while (!mbar_try_wait(BAR_U_FULL(v % US), (v / US) & 1) && clock64() - t0 < kWaitLimitCycles) {
           }
         }
       }
@@ -323,47 +351,62 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       const uint32_t idesc_id = make_idesc(Pack16<T>::kFmt, 16);
       const uint32_t idesc_ug = make_idesc(1, NS);
       const uint64_t desc_id = make_desc(smem_u32(ident), 32);
-      const uint64_t desc_ghi = make_desc(smem_u32(g_hi), ROWB);
-      const uint64_t desc_glo = make_desc(smem_u32(g_lo), ROWB);
-      int t = 0, item_no = 0;
+      int t = 0, rb = 0, item_no = 0;
       bool ok = true;
       for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x, ++item_no) {
         const WorkItem w = p.items[it];
         if (!mbar_wait<true>(BAR_G, item_no & 1, abort_flag, error, 3)) break;
         tc_fence_after();
         const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
-        const int nbox = (w.ncols + 63) / 64;
-        for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
-          const int s = t % S, b = t % NACC;
-          if (!mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
-          if (t >= NACC && !mbar_wait<true>(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sbase = smem_u32(stage_base + s * Cfg::STAGE_BYTES);
-          const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
-          // theta -> fp32, 16 columns at a time
-          for (int c = 0; c < nbox; ++c)
+        const int nsub = (w.ncols + NS - 1) / NS;
+        for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128, ++rb) {
+          const int u = rb % US;
+          if (!mbar_wait<true>(BAR_U_FULL(u), (rb / US) & 1, abort_flag, error, 9)) { ok = false; break; }
+          const uint32_t uhi = smem_u32(u_base + u * 2 * Cfg::U_BYTES), ulo = uhi + Cfg::U_BYTES;
+          for (int sub = 0; sub < nsub; ++sub, ++t) {
+            const int s = t % S, b = t % NACC;
+            if (!mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
+            if (t >= NACC && !mbar_wait<true>(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sbase = smem_u32(theta_base + s * Cfg::THETA_BYTES);
+            const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
+            const int nbox = (min(NS, w.ncols - NS * sub) + 63) / 64;
+            // theta -> fp32, 16 columns at a time
+            for (int c = 0; c < nbox; ++c)
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma(d + static_cast<uint32_t>(64 * c + 16 * k), make_desc(sbase + c * 16384 + 32 * k, 128), desc_id, idesc_id, 0u);
-          // + c b U G, split operands
-          const uint32_t uhi = sbase + Cfg::THETA_BYTES, ulo = uhi + Cfg::U_BYTES;
+              for (int k = 0; k < 4; ++k)
+                umma(d + static_cast<uint32_t>(64 * c + 16 * k), make_desc(sbase + c * 16384 + 32 * k, 128), desc_id, idesc_id, 0u);
+            // + c b U G, split operands
+            const uint64_t desc_ghi = make_desc(smem_u32(g_base + sub * 2 * Cfg::G_BYTES), ROWB);
+            const uint64_t desc_glo = make_desc(smem_u32(g_base + sub * 2 * Cfg::G_BYTES + Cfg::G_BYTES), ROWB);
 #pragma unroll
-          for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(ulo + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+            for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(ulo + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
 #pragma unroll
-          for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_glo + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+            for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_glo + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
 #pragma unroll
-          for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
-          umma_commit(BAR_ACC_FULL(b));
+            for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+            umma_commit(BAR_ACC_FULL(b));
+          }
+          if (ok) umma_commit(BAR_U_FREE(u));   // arrives once every product that reads this U tile has completed
         }
       }
     }
   } else {
     // ===================================== epilogue warps =====================================
+    // Two groups of eight warps take alternate tiles, so that one group computes while the other
+    // waits for an accumulator, reads tensor memory or hands its tile over.  Inside a group, warp
+    // (quad, half) owns rows 32 quad .. 32 quad + 31 and columns 64 half .. 64 half + 63 of the tile.
     const int e = warp - 2;                 // 0..15
+    const int grp = e >> 3;                 // tile parity served by this warp
     const int quad = warp & 3;              // tensor-memory lane quadrant this warp may read
-    const int cgrp = e >> 2;                // which group of COLS_PER_WARP columns
+    const int half = (e >> 2) & 1;          // which 64 columns (= which TMA box) of the tile
     const int et = e * 32 + lane;           // 0..511
-    constexpr int CPW = Cfg::COLS_PER_WARP;
+    const uint32_t tmem_warp = tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(64 * half);
+    const int row_in_tile = 32 * quad + lane;
+    const uint32_t row_xor = static_cast<uint32_t>(row_in_tile & 7);
+    const uint32_t out_off = static_cast<uint32_t>(half * 16384 + row_in_tile * 128);
+    const uint32_t theta_s32 = smem_u32(theta_base);
+    const uint32_t g_s32 = smem_u32(g_base);
     int t = 0, item_no = 0;
     bool ok = true;
     for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x, ++item_no) {
@@ -371,11 +414,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       const TensorDesc& td = p.tensors[w.tensor];
       const uint32_t tid = static_cast<uint32_t>(td.id);
       const int r = td.rank;
-      // ---- coefficient strip c b G -> K-major hi/lo operands (all MMAs of the previous item are
-      //      complete: this warp has waited for the accumulator of its last tile) ----
-      for (int idx = et; idx < (KP / 2) * (NS / 8); idx += kEpiWarps * 32) {
-        const int kp = idx / (NS / 8), o = idx % (NS / 8);
-        const int cc = 8 * o;
+      // The coefficient strips may be overwritten once every product of the previous item has
+      // completed, i.e. once the accumulator of its last tile is full (that tile may belong to the other group).
+      if (t > 0 && !mbar_wait<false>(BAR_ACC_FULL((t - 1) % NACC), ((t - 1) / NACC) & 1, abort_flag, error, 10)) break;
+      // ---- coefficient strips c b G -> K-major hi/lo operands, one per tile of a row block ----
+      for (int idx = et; idx < (KP / 2) * (NSUB * NS / 8); idx += kEpiWarps * 32) {
+        const int kp = idx / (NSUB * NS / 8), o = idx % (NSUB * NS / 8);
+        const int cc = 8 * o;                       // column within the item's strip
+        if (cc >= ((w.ncols + NS - 1) / NS) * NS) continue;   // tiles of this item that do not exist
         float g0[8], g1[8];
         if (cc < w.ncols && 2 * kp < r) {
           coeffs8<BITS, false>(td, p.keys, p.unit, p.cb, 2 * kp, w.col0 + cc, g0);
@@ -389,13 +435,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
 #pragma unroll
           for (int i = 0; i < 8; ++i) g1[i] = 0.0f;
         }
+        const uint32_t g_hi = g_s32 + static_cast<uint32_t>((cc / NS) * 2 * Cfg::G_BYTES);
+        const uint32_t g_lo = g_hi + static_cast<uint32_t>(Cfg::G_BYTES);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           uint32_t hi, lo;
           split_bf16(g0[i], g1[i], hi, lo);
-          const uint32_t off = swizzle(static_cast<uint32_t>((cc + i) * ROWB + 4 * kp), ROWB);
-          *reinterpret_cast<uint32_t*>(g_hi + off) = hi;
-          *reinterpret_cast<uint32_t*>(g_lo + off) = lo;
+          const uint32_t off = swizzle(static_cast<uint32_t>(((cc % NS) + i) * ROWB + 4 * kp), ROWB);
+          sts32(g_hi + off, hi);
+          sts32(g_lo + off, lo);
         }
       }
       fence_proxy_async();
@@ -403,46 +451,47 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       if (lane == 0) mbar_arrive(BAR_G);
 
       const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
-      const bool active = cgrp * CPW < w.ncols;
-      static_assert(CPW == 32, "the epilogue below handles 32 columns per warp");
-      const uint32_t tmem_warp = tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(cgrp * CPW);
-      for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end; row0 += 128, ++t) {
-        const int s = t % S, b = t % NACC;
-        if (!mbar_wait<false>(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
-        tc_fence_after();
-        if (active) {
-          const int row_in_tile = 32 * quad + lane;
-          const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
-          // number of this thread's first octet in the tensor (element index / 8)
-          const uint64_t oct0 = (static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + cgrp * CPW)) >> 3;
-          const uint32_t oct0_lo = static_cast<uint32_t>(oct0), oct0_hi = static_cast<uint32_t>(oct0 >> 32);
-          // output position: box (col / 64), row, 16-byte chunk XOR-swizzled with the row
-          uint8_t* out_box = stage_base + s * Cfg::STAGE_BYTES + ((cgrp * CPW) >> 6) * 16384 + row_in_tile * 128;
-          const uint32_t chunk0 = static_cast<uint32_t>(((cgrp * CPW) & 63) >> 3);
-          const uint32_t row_xor = static_cast<uint32_t>(row_in_tile & 7);
-          uint32_t h0[16], h1[16];
-          tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS), h0);
-          tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 16), h1);
-          tmem_ld_wait();
-          // four octets per thread, kept independent so that their generator chains interleave
+      const int nsub = (w.ncols + NS - 1) / NS;
+      for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128) {
+        const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
+        const uint64_t row_e = static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + 64 * half);
+        for (int sub = 0; sub < nsub; ++sub, ++t) {
+          if ((t & 1) != grp) continue;             // the other group's tile
+          const int s = t % S, b = t % NACC;
+          if (!mbar_wait<false>(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
+          tc_fence_after();
+          if (NS * sub + 64 * half < w.ncols) {
+            // number of this thread's first octet in the tensor (element index / 8)
+            const uint64_t oct0 = (row_e + static_cast<uint64_t>(NS * sub)) >> 3;
+            const uint32_t oct0_lo = static_cast<uint32_t>(oct0), oct0_hi = static_cast<uint32_t>(oct0 >> 32);
+            const uint32_t out_box = theta_s32 + static_cast<uint32_t>(s * Cfg::THETA_BYTES) + out_off;   // shared-space address
+#pragma unroll 1
+            for (int part = 0; part < 2; ++part) {   // 32 columns at a time
+              uint32_t h0[16], h1[16];
+              tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 32 * part), h0);
+              tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 32 * part + 16), h1);
+              tmem_ld_wait();
+              // four octets per thread, kept independent so that their generator chains interleave
 #pragma unroll
-          for (int o = 0; o < 4; ++o) {
-            float acc[8];
+              for (int o = 0; o < 4; ++o) {
+                float acc[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
-            const uint32_t lo = oct0_lo + static_cast<uint32_t>(o);
-            normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, acc);
-            const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
-                                       Pack16<T>::pack(acc[6], acc[7]));
-            *reinterpret_cast<uint4*>(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4)) = q;
+                for (int i = 0; i < 8; ++i) acc[i] = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
+                const uint32_t lo = oct0_lo + static_cast<uint32_t>(4 * part + o);
+                normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, acc);
+                const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
+                                           Pack16<T>::pack(acc[6], acc[7]));
+                sts128(out_box + ((static_cast<uint32_t>(4 * part + o) ^ row_xor) << 4), q);
+              }
+            }
           }
-        }
-        tc_fence_before();
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(BAR_ACC_EMPTY(b));
-          mbar_arrive(BAR_OUT(s));
+          tc_fence_before();
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(BAR_ACC_EMPTY(b));
+            mbar_arrive(BAR_OUT(s));
+          }
         }
       }
     }
@@ -474,7 +523,7 @@ __global__ void split_subspace_rowmajor_kernel(const float* __restrict__ U, int6
 size_t umma_smem_bytes(int kpad) {
   return kpad == 16 ? UmmaCfg<16>::SMEM_BYTES : (kpad == 32 ? UmmaCfg<32>::SMEM_BYTES : UmmaCfg<64>::SMEM_BYTES);
 }
-int umma_strip_cols(int kpad) { (void)kpad; return 128; }
+int umma_strip_cols(int kpad) { return kpad == 64 ? UmmaCfg<64>::NS * UmmaCfg<64>::NSUB : (kpad == 32 ? UmmaCfg<32>::NS * UmmaCfg<32>::NSUB : UmmaCfg<16>::NS * UmmaCfg<16>::NSUB); }
 
 namespace {
 template <typename T, int BITS>
