@@ -34,6 +34,25 @@ METRIC = "zgr_step_params_per_sec"
 UNIT = "params/s"
 
 
+# DRAM traffic per launch of the dominant kernel from one ncu capture (profiles/sweep_umma_bf16_k32_llama7b.md:
+# small case, scaled by the elements processed), valid only for the kernel source it was taken from.
+NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.77e9,
+               "source": "paper_2601_12917_b200/csrc/zgr_umma.cu", "sha1": "d029020ee4dde7373aaab4872efc63e8a7224a62"}
+
+
+def ncu_traffic(kernel: str, workload: str):
+    import hashlib
+    if kernel != NCU_TRAFFIC["kernel"] or workload != NCU_TRAFFIC["workload"]:
+        return None
+    try:
+        with open(os.path.join(ROOT, NCU_TRAFFIC["source"]), "rb") as f:
+            if hashlib.sha1(f.read()).hexdigest() != NCU_TRAFFIC["sha1"]:
+                return None           # the kernel has changed since the counters were taken
+    except OSError:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"]
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -74,7 +93,7 @@ def cpu_baseline(wl, bits: int):
     rows = 4096 if wl.params > (1 << 28) else 1024
     sweeps_per_step = 3 * wl.queries
     secs, n, threads, what = oracle_sample(wl, rows, 1, bits)       # also the warm-up
-    reps = int(min(24, max(1, round(10.0 / max(secs * threads, 1e-3)))))
+    reps = int(min(48, max(1, round(15.0 / max(secs * threads, 1e-3)))))
     secs, n, threads, what = oracle_sample(wl, rows, reps, bits)
     return {"value": n * reps / secs / sweeps_per_step, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"{reps} sweeps over a {what} in {secs:.2f} s, scaled by 1/{sweeps_per_step} sweeps per step"}
@@ -255,8 +274,10 @@ def main():
     if top:
         per_launch_ms = top["ms_total"] / top["launches"]
         achieved = 2 * eb * top["elements"] / (per_launch_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
-                    "peak_kind": f"of {peak_kind}", "kernel": f"sweep_{top['path']}_kernel(k={top['kpad']})", "launches": top["launches"],
+        kname = f"sweep_{top['path']}_kernel(k={top['kpad']})"
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": ncu_traffic(kname, wl.name) if args.layers is None else None,
+                    "peak_kind": f"of {peak_kind}", "kernel": kname, "launches": top["launches"],
                     "ms_per_launch": per_launch_ms, "algorithmic_bytes_per_launch": 2 * eb * top["elements"],
                     "share_of_kernel_time": top["ms_total"] / sum(k["ms_total"] for k in kernels)}
 
