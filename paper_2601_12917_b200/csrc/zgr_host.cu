@@ -44,7 +44,8 @@ struct zgr_ctx {
   bool descs_dirty = false;
   std::vector<void*> owned;           // device allocations made by the library
   std::vector<Group> groups;          // sweep plan
-  std::vector<WorkItem> stats_items;  // plan of the norm kernel
+  std::vector<WorkItem> stats_items;  // plan of the norm kernel (tensors not served by the tcgen05 kernel)
+  bool stats_planned = false;
   WorkItem* d_stats_items = nullptr;
   double* d_stats = nullptr;
   bool active = false;
@@ -471,12 +472,13 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
   const size_t n = ctx->descs.size();
-  if (ctx->stats_items.empty()) {
-    // generic tiling of every tensor: strips of 64 columns
+  if (!ctx->stats_planned) {
+    // tensors served by the tcgen05 kernel reuse its work items; all others get a generic tiling (strips of 64 columns)
     int64_t total = ctx->d;
     int64_t target = std::min<int64_t>(std::max<int64_t>(total / (static_cast<int64_t>(ctx->sm_count) * 64), 4096), 131072);
     for (size_t l = 0; l < n; ++l) {
       const TensorDesc& t = ctx->descs[l];
+      if (t.umma && ctx->b != 0.0) continue;
       for (int64_t c0 = 0; c0 < t.cols; c0 += 64) {
         const int ncols = static_cast<int>(std::min<int64_t>(64, t.cols - c0));
         const int64_t nrows = std::max<int64_t>(1, target / ncols);
@@ -484,10 +486,13 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
           ctx->stats_items.push_back(WorkItem{static_cast<int32_t>(l), ncols, r0, std::min(nrows, t.rows - r0), c0});
       }
     }
-    rc = dev_alloc(ctx, &ctx->d_stats_items, ctx->stats_items.size());
-    if (rc == ZGR_OK)
-      rc = check(ctx, cudaMemcpy(ctx->d_stats_items, ctx->stats_items.data(), ctx->stats_items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
-    if (rc != ZGR_OK) return rc;
+    if (!ctx->stats_items.empty()) {
+      rc = dev_alloc(ctx, &ctx->d_stats_items, ctx->stats_items.size());
+      if (rc == ZGR_OK)
+        rc = check(ctx, cudaMemcpy(ctx->d_stats_items, ctx->stats_items.data(), ctx->stats_items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
+      if (rc != ZGR_OK) return rc;
+    }
+    ctx->stats_planned = true;
   }
   rc = check(ctx, cudaMemsetAsync(ctx->d_stats, 0, 3 * n * sizeof(double), st));
   if (rc != ZGR_OK) return rc;
@@ -500,10 +505,20 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
   p.n_items = static_cast<int32_t>(ctx->stats_items.size());
   p.cb = static_cast<float>(ctx->b);
   p.stats = ctx->d_stats;
-  const int grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * 4));
-  rc = check(ctx, launch_stats(ctx->cfg.bits_per_normal, p, grid, st));
-  if (rc != ZGR_OK) return rc;
-  ctx->launches++;
+  if (p.n_items > 0) {
+    const int grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * 4));
+    rc = check(ctx, launch_stats(ctx->cfg.bits_per_normal, p, grid, st));
+    if (rc != ZGR_OK) return rc;
+    ctx->launches++;
+  }
+  for (const Group& g : ctx->groups) {
+    if (g.kc.path != PATH_UMMA || g.items.empty()) continue;
+    p.items = g.d_items;
+    p.n_items = static_cast<int32_t>(g.items.size());
+    rc = check(ctx, launch_stats_umma(g.kc, p, ctx->d_tmaps, ctx->d_err, g.grid, st));
+    if (rc != ZGR_OK) return rc;
+    ctx->launches++;
+  }
   rc = check(ctx, cudaMemcpyAsync(out, ctx->d_stats, 3 * n * sizeof(double), cudaMemcpyDeviceToHost, st));
   if (rc != ZGR_OK) return rc;
   return check(ctx, cudaStreamSynchronize(st));

@@ -30,6 +30,7 @@ cudaError_t launch_sweep(const KernelChoice& kc, const SweepParams& p, int grid,
 int umma_strip_cols(int kpad);
 size_t umma_smem_bytes(int kpad);
 cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
+cudaError_t launch_stats_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
 cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st);
 
 cudaError_t launch_stats(int bits, const SweepParams& p, int grid, cudaStream_t st);

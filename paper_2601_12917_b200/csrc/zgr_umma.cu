@@ -221,7 +221,10 @@ struct TileCoord {
 // Work item = NSUB adjacent column tiles (a strip of up to 128*NSUB columns) x a range of rows.
 // Tiles are visited row block by row block, the NSUB tiles of a row block one after the other, so
 // that a CTA touches up to 256*NSUB contiguous bytes of every row and loads each U tile once.
-template <typename T, int BITS, int KP>
+// STATS = true turns the same pipeline into the norm bookkeeping: no weights are loaded or stored,
+// D = b U G only, and the epilogue accumulates sum (a Z)^2, sum (b U G)^2 and sum z^2 per tensor
+// (p.iso carries the scale a, p.cb = b, p.stats the three doubles per tensor).
+template <typename T, int BITS, int KP, bool STATS = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
                                                                      int* __restrict__ error) {
   using Cfg = UmmaCfg<KP>;
@@ -306,7 +309,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
           mbar_arrive_expect_tx(BAR_U_FULL(u), static_cast<uint32_t>(2 * Cfg::U_BYTES));
           tma_load_2d(udst, tm + 1, 0, row0, BAR_U_FULL(u));
           tma_load_2d(udst + Cfg::U_BYTES, tm + 2, 0, row0, BAR_U_FULL(u));
-          for (int sub = 0; sub < nsub; ++sub, ++t) {
+          for (int sub = 0; sub < nsub && !STATS; ++sub, ++t) {
             const int s = t % S;
             if (t >= S) {
               // the epilogue has written tile t-S into this stage: store it, then the stage is free
@@ -326,7 +329,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       }
       // drain: store the last tiles
       const int total = t;
-      for (int v = (total > S ? total - S : 0); v < total && ok; ++v) {
+      for (int v = (total > S ? total - S : 0); v < total && ok && !STATS; ++v) {
         if (!mbar_wait<true>(BAR_OUT(v % S), (v / S) & 1, abort_flag, error, 2)) { ok = false; break; }
         store_tile(v % S);
       }
@@ -365,14 +368,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
           const uint32_t uhi = smem_u32(u_base + u * 2 * Cfg::U_BYTES), ulo = uhi + Cfg::U_BYTES;
           for (int sub = 0; sub < nsub; ++sub, ++t) {
             const int s = t % S, b = t % NACC;
-            if (!mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
+            if (!STATS && !mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
             if (t >= NACC && !mbar_wait<true>(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
             tc_fence_after();
             const uint32_t sbase = smem_u32(theta_base + s * Cfg::THETA_BYTES);
             const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
             const int nbox = (min(NS, w.ncols - NS * sub) + 63) / 64;
             // theta -> fp32, 16 columns at a time
-            for (int c = 0; c < nbox; ++c)
+            for (int c = 0; c < nbox && !STATS; ++c)
 #pragma unroll
               for (int k = 0; k < 4; ++k)
                 umma(d + static_cast<uint32_t>(64 * c + 16 * k), make_desc(sbase + c * 16384 + 32 * k, 128), desc_id, idesc_id, 0u);
@@ -380,7 +383,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
             const uint64_t desc_ghi = make_desc(smem_u32(g_base + sub * 2 * Cfg::G_BYTES), ROWB);
             const uint64_t desc_glo = make_desc(smem_u32(g_base + sub * 2 * Cfg::G_BYTES + Cfg::G_BYTES), ROWB);
 #pragma unroll
-            for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(ulo + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+            for (int k = 0; k < KP / 16; ++k)
+              umma(d, make_desc(ulo + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, (STATS && k == 0) ? 0u : 1u);
 #pragma unroll
             for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_glo + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
 #pragma unroll
@@ -452,6 +456,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
 
       const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
       const int nsub = (w.ncols + NS - 1) / NS;
+      double sum_iso = 0.0, sum_gd = 0.0, sum_z = 0.0;   // STATS only
       for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128) {
         const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
         const uint64_t row_e = static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + 64 * half);
@@ -471,6 +476,30 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
               tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 32 * part), h0);
               tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 32 * part + 16), h1);
               tmem_ld_wait();
+              if constexpr (STATS) {
+                float f_iso = 0.0f, f_gd = 0.0f, f_z = 0.0f;
+#pragma unroll
+                for (int o = 0; o < 4; ++o) {
+                  float zi[8];
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) zi[i] = 0.0f;
+                  const uint32_t lo = oct0_lo + static_cast<uint32_t>(4 * part + o);
+                  normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, zi);
+                  const bool live = row < row_end && NS * sub + 64 * half + 32 * part + 8 * o < w.ncols;
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) {
+                    const float gd = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
+                    if (live) {
+                      f_iso = fmaf(zi[i], zi[i], f_iso);
+                      f_gd = fmaf(gd, gd, f_gd);
+                      f_z = fmaf(zi[i] + gd, zi[i] + gd, f_z);
+                    }
+                  }
+                }
+                sum_iso += static_cast<double>(f_iso);
+                sum_gd += static_cast<double>(f_gd);
+                sum_z += static_cast<double>(f_z);
+              } else {
               // four octets per thread, kept independent so that their generator chains interleave
 #pragma unroll
               for (int o = 0; o < 4; ++o) {
@@ -483,6 +512,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
                                            Pack16<T>::pack(acc[6], acc[7]));
                 sts128(out_box + ((static_cast<uint32_t>(4 * part + o) ^ row_xor) << 4), q);
               }
+              }
             }
           }
           tc_fence_before();
@@ -490,8 +520,21 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
           __syncwarp();
           if (lane == 0) {
             mbar_arrive(BAR_ACC_EMPTY(b));
-            mbar_arrive(BAR_OUT(s));
+            if (!STATS) mbar_arrive(BAR_OUT(s));
           }
+        }
+      }
+      if constexpr (STATS) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          sum_iso += __shfl_xor_sync(0xFFFFFFFFu, sum_iso, off);
+          sum_gd += __shfl_xor_sync(0xFFFFFFFFu, sum_gd, off);
+          sum_z += __shfl_xor_sync(0xFFFFFFFFu, sum_z, off);
+        }
+        if (lane == 0) {
+          atomicAdd(p.stats + 3 * w.tensor + 0, sum_iso);
+          atomicAdd(p.stats + 3 * w.tensor + 1, sum_gd);
+          atomicAdd(p.stats + 3 * w.tensor + 2, sum_z);
         }
       }
     }
@@ -526,11 +569,11 @@ size_t umma_smem_bytes(int kpad) {
 int umma_strip_cols(int kpad) { return kpad == 64 ? UmmaCfg<64>::NS * UmmaCfg<64>::NSUB : (kpad == 32 ? UmmaCfg<32>::NS * UmmaCfg<32>::NSUB : UmmaCfg<16>::NS * UmmaCfg<16>::NSUB); }
 
 namespace {
-template <typename T, int BITS>
+template <typename T, int BITS, bool STATS = false>
 cudaError_t launch_umma_kp(int kpad, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
 #define ZGR_LAUNCH_UMMA(KPV)                                                                                       \
   {                                                                                                                \
-    auto k = sweep_umma_kernel<T, BITS, KPV>;                                                                      \
+    auto k = sweep_umma_kernel<T, BITS, KPV, STATS>;                                                                 \
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<KPV>::SMEM_BYTES); \
     if (e != cudaSuccess) return e;                                                                                \
     k<<<grid, kUmmaThreads, UmmaCfg<KPV>::SMEM_BYTES, st>>>(p, tmaps, error);                                      \
@@ -552,6 +595,12 @@ cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, cons
     return kc.bits == 32 ? launch_umma_kp<__half, 32>(kc.kpad, p, tmaps, error, grid, st) : launch_umma_kp<__half, 16>(kc.kpad, p, tmaps, error, grid, st);
   }
   return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_stats_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
+  // the storage type plays no role when no weights are touched: one instantiation serves all
+  return kc.bits == 32 ? launch_umma_kp<__nv_bfloat16, 32, true>(kc.kpad, p, tmaps, error, grid, st)
+                       : launch_umma_kp<__nv_bfloat16, 16, true>(kc.kpad, p, tmaps, error, grid, st);
 }
 
 cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st) {

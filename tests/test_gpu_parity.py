@@ -271,7 +271,8 @@ def test_restore_is_within_two_ulp_at_lr_zero():
 # ------------------------------------------------------------------------------------- norms
 @pytest.mark.parametrize("bits", [32, 16])
 def test_norm_bookkeeping(bits):
-    shapes, ranks = [(64, 256), (1, 100), (40, 72), (48, 128)], [8, 0, 3, 16]
+    # tensor-core tensors (ragged row blocks and strips included), CUDA-core, isotropic and fallback tensors
+    shapes, ranks = [(64, 256), (1, 100), (40, 72), (48, 128), (300, 392), (130, 1032), (45, 100)], [8, 0, 3, 16, 32, 64, 20]
     p = Pair(shapes, ranks, "bf16", bits=bits, alpha=0.4)
     got = p.lib.get_stats(17)
     for l in range(len(shapes)):
