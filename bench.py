@@ -37,7 +37,7 @@ UNIT = "params/s"
 # DRAM traffic per launch of the dominant kernel from one ncu capture (profiles/sweep_umma_bf16_k32_llama7b.md:
 # small case, scaled by the elements processed), valid only for the kernel source it was taken from.
 NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.77e9,
-               "source": "paper_2601_12917_b200/csrc/zgr_umma.cu", "sha1": "7272f9d5fc36210a6ce73ffe709dd90c174beda1"}
+               "source": "paper_2601_12917_b200/csrc/zgr_umma.cu", "sha1": "32fd37079633d0ec5c0ed9fdc10071367403bf7d"}
 
 
 def ncu_traffic(kernel: str, workload: str):

@@ -252,11 +252,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(BAR_FULL(s), 1);
-      mbar_init(BAR_OUT(s), kEpiWarps / 2);
+      mbar_init(BAR_OUT(s), kEpiWarps);
     }
     for (int b = 0; b < NACC; ++b) {
       mbar_init(BAR_ACC_FULL(b), 1);
-      mbar_init(BAR_ACC_EMPTY(b), kEpiWarps / 2);
+      mbar_init(BAR_ACC_EMPTY(b), kEpiWarps);
     }
     for (int u = 0; u < US; ++u) {
       mbar_init(BAR_U_FULL(u), 1);
@@ -397,18 +397,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
     }
   } else {
     // ===================================== epilogue warps =====================================
-    // Two groups of eight warps take alternate tiles, so that one group computes while the other
-    // waits for an accumulator, reads tensor memory or hands its tile over.  Inside a group, warp
-    // (quad, half) owns rows 32 quad .. 32 quad + 31 and columns 64 half .. 64 half + 63 of the tile.
+    // Warp (quad, cgrp) owns rows 32 quad .. 32 quad + 31 and columns 32 cgrp .. 32 cgrp + 31 of every tile.
     const int e = warp - 2;                 // 0..15
-    const int grp = e >> 3;                 // tile parity served by this warp
     const int quad = warp & 3;              // tensor-memory lane quadrant this warp may read
-    const int half = (e >> 2) & 1;          // which 64 columns (= which TMA box) of the tile
-    const int et = e * 32 + lane;           // 0..511
-    const uint32_t tmem_warp = tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(64 * half);
+    const int cgrp = e >> 2;                // which 32 columns of the tile
+    const int et = e * 32 + lane;
+    const uint32_t tmem_warp = tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(32 * cgrp);
     const int row_in_tile = 32 * quad + lane;
     const uint32_t row_xor = static_cast<uint32_t>(row_in_tile & 7);
-    const uint32_t out_off = static_cast<uint32_t>(half * 16384 + row_in_tile * 128);
+    const uint32_t chunk0 = static_cast<uint32_t>(((32 * cgrp) & 63) >> 3);
+    const uint32_t out_off = static_cast<uint32_t>(((32 * cgrp) >> 6) * 16384 + row_in_tile * 128);
     const uint32_t theta_s32 = smem_u32(theta_base);
     const uint32_t g_s32 = smem_u32(g_base);
     int t = 0, item_no = 0;
@@ -418,9 +416,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       const TensorDesc& td = p.tensors[w.tensor];
       const uint32_t tid = static_cast<uint32_t>(td.id);
       const int r = td.rank;
-      // The coefficient strips may be overwritten once every product of the previous item has
-      // completed, i.e. once the accumulator of its last tile is full (that tile may belong to the other group).
-      if (t > 0 && !mbar_wait<false>(BAR_ACC_FULL((t - 1) % NACC), ((t - 1) / NACC) & 1, abort_flag, error, 10)) break;
       // ---- coefficient strips c b G -> K-major hi/lo operands, one per tile of a row block ----
       for (int idx = et; idx < (KP / 2) * (NSUB * NS / 8); idx += kEpiWarps * 32) {
         const int kp = idx / (NSUB * NS / 8), o = idx % (NSUB * NS / 8);
@@ -459,60 +454,55 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       double sum_iso = 0.0, sum_gd = 0.0, sum_z = 0.0;   // STATS only
       for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128) {
         const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
-        const uint64_t row_e = static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + 64 * half);
+        const uint64_t row_e = static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + 32 * cgrp);
         for (int sub = 0; sub < nsub; ++sub, ++t) {
-          if ((t & 1) != grp) continue;             // the other group's tile
           const int s = t % S, b = t % NACC;
           if (!mbar_wait<false>(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
           tc_fence_after();
-          if (NS * sub + 64 * half < w.ncols) {
-            // number of this thread's first octet in the tensor (element index / 8)
+          if (NS * sub + 32 * cgrp < w.ncols) {
             const uint64_t oct0 = (row_e + static_cast<uint64_t>(NS * sub)) >> 3;
             const uint32_t oct0_lo = static_cast<uint32_t>(oct0), oct0_hi = static_cast<uint32_t>(oct0 >> 32);
-            const uint32_t out_box = theta_s32 + static_cast<uint32_t>(s * Cfg::THETA_BYTES) + out_off;   // shared-space address
-#pragma unroll 1
-            for (int part = 0; part < 2; ++part) {   // 32 columns at a time
-              uint32_t h0[16], h1[16];
-              tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 32 * part), h0);
-              tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 32 * part + 16), h1);
-              tmem_ld_wait();
-              if constexpr (STATS) {
-                float f_iso = 0.0f, f_gd = 0.0f, f_z = 0.0f;
-#pragma unroll
-                for (int o = 0; o < 4; ++o) {
-                  float zi[8];
-#pragma unroll
-                  for (int i = 0; i < 8; ++i) zi[i] = 0.0f;
-                  const uint32_t lo = oct0_lo + static_cast<uint32_t>(4 * part + o);
-                  normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, zi);
-                  const bool live = row < row_end && NS * sub + 64 * half + 32 * part + 8 * o < w.ncols;
-#pragma unroll
-                  for (int i = 0; i < 8; ++i) {
-                    const float gd = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
-                    if (live) {
-                      f_iso = fmaf(zi[i], zi[i], f_iso);
-                      f_gd = fmaf(gd, gd, f_gd);
-                      f_z = fmaf(zi[i] + gd, zi[i] + gd, f_z);
-                    }
-                  }
-                }
-                sum_iso += static_cast<double>(f_iso);
-                sum_gd += static_cast<double>(f_gd);
-                sum_z += static_cast<double>(f_z);
-              } else {
-              // four octets per thread, kept independent so that their generator chains interleave
+            const uint32_t out_box = theta_s32 + static_cast<uint32_t>(s * Cfg::THETA_BYTES) + out_off;
+            uint32_t h0[16], h1[16];
+            tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS), h0);
+            tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 16), h1);
+            tmem_ld_wait();
+            if constexpr (STATS) {
+              float f_iso = 0.0f, f_gd = 0.0f, f_z = 0.0f;
 #pragma unroll
               for (int o = 0; o < 4; ++o) {
-                float acc[8];
+                float zi[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) acc[i] = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
-                const uint32_t lo = oct0_lo + static_cast<uint32_t>(4 * part + o);
-                normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, acc);
-                const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
-                                           Pack16<T>::pack(acc[6], acc[7]));
-                sts128(out_box + ((static_cast<uint32_t>(4 * part + o) ^ row_xor) << 4), q);
+                for (int i = 0; i < 8; ++i) zi[i] = 0.0f;
+                const uint32_t lo = oct0_lo + static_cast<uint32_t>(o);
+                normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, zi);
+                const bool live = row < row_end && NS * sub + 32 * cgrp + 8 * o < w.ncols;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const float gd = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
+                  if (live) {
+                    f_iso = fmaf(zi[i], zi[i], f_iso);
+                    f_gd = fmaf(gd, gd, f_gd);
+                    f_z = fmaf(zi[i] + gd, zi[i] + gd, f_z);
+                  }
+                }
               }
-              }
+              sum_iso += static_cast<double>(f_iso);
+              sum_gd += static_cast<double>(f_gd);
+              sum_z += static_cast<double>(f_z);
+            } else {
+            // four octets per thread, kept independent so that their generator chains interleave
+#pragma unroll
+            for (int o = 0; o < 4; ++o) {
+              float acc[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) acc[i] = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
+              const uint32_t lo = oct0_lo + static_cast<uint32_t>(o);
+              normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, acc);
+              const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
+                                         Pack16<T>::pack(acc[6], acc[7]));
+              sts128(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4), q);
+            }
             }
           }
           tc_fence_before();
