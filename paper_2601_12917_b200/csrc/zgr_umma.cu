@@ -34,8 +34,6 @@
 namespace zgr {
 namespace {
 
-constexpr int kEpiWarps = 16;
-constexpr int kUmmaThreads = 32 * (2 + kEpiWarps);
 constexpr unsigned long long kWaitLimitCycles = 4000000000ull;  // ~2 s at 2 GHz
 
 // ---------------------------------------------------------------------------------------------
@@ -190,13 +188,42 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
+// Tile configuration per contraction width.  TILE_N = 192 runs 24 epilogue warps on 128 x 192 tiles
+// (three 64-column boxes); TILE_N = 128 runs 16 on 128 x 128 tiles.
+#ifndef ZGR_TILE_N16
+#define ZGR_TILE_N16 128
+#endif
+#ifndef ZGR_TILE_N32
+#define ZGR_TILE_N32 128
+#endif
+#ifndef ZGR_S16
+#define ZGR_S16 4
+#endif
+#ifndef ZGR_S32
+#define ZGR_S32 4
+#endif
+#ifndef ZGR_S64
+#define ZGR_S64 4
+#endif
+#ifndef ZGR_N16
+#define ZGR_N16 4
+#endif
+#ifndef ZGR_N32
+#define ZGR_N32 3
+#endif
+#ifndef ZGR_N64
+#define ZGR_N64 1
+#endif
 template <int KP>
 struct UmmaCfg {
-  static constexpr int NS = 128;                           // columns per tile / per accumulator buffer
-  static constexpr int NSUB = KP == 64 ? 1 : (KP == 32 ? 2 : 4);   // adjacent tiles per row block that share one U tile
-  static constexpr int STAGES = KP == 64 ? 4 : 5;          // theta tiles in flight (loaded, transformed in place, stored)
+  static constexpr int NS = KP == 64 ? 128 : (KP == 32 ? ZGR_TILE_N32 : ZGR_TILE_N16);   // columns per tile / per accumulator buffer
+  static constexpr bool WIDE = NS > 128;
+  static constexpr int EPI_WARPS = NS / 8;                 // one epilogue warp per 32 rows x 32 columns of a tile
+  static constexpr int THREADS = 32 * (2 + EPI_WARPS);
+  static constexpr int NSUB = KP == 64 ? ZGR_N64 : (KP == 32 ? ZGR_N32 : ZGR_N16);   // adjacent tiles per row block that share one U tile
+  static constexpr int STAGES = KP == 64 ? ZGR_S64 : (KP == 32 ? ZGR_S32 : ZGR_S16);  // theta tiles in flight (loaded, transformed in place, stored)
   static constexpr int USTAGES = 2;                        // U tiles in flight
-  static constexpr int NACC = 4;                           // accumulator buffers in tensor memory
+  static constexpr int NACC = WIDE ? 2 : 4;                // accumulator buffers in tensor memory
   static constexpr int ROWB = KP * 2;                      // bytes per row of the U and G operands
   static constexpr int THETA_BYTES = 128 * NS * 2;         // NS/64 boxes of 128 rows x 128 B
   static constexpr int U_BYTES = 128 * ROWB;               // one of hi / lo
@@ -205,7 +232,7 @@ struct UmmaCfg {
   static constexpr int BAR_BYTES = 1024;
   static constexpr int SMEM_BYTES =
       STAGES * THETA_BYTES + USTAGES * 2 * U_BYTES + NSUB * 2 * G_BYTES + ID_BYTES + BAR_BYTES + 1024 /* alignment slack */;
-  static constexpr int TMEM_COLS = NACC * NS;
+  static constexpr int TMEM_COLS = NACC * NS <= 256 ? 256 : 512;   // allocations are powers of two
   static_assert(SMEM_BYTES <= 232448, "shared-memory budget of one CTA");
 };
 
@@ -225,10 +252,11 @@ struct TileCoord {
 // D = b U G only, and the epilogue accumulates sum (a Z)^2, sum (b U G)^2 and sum z^2 per tensor
 // (p.iso carries the scale a, p.cb = b, p.stats the three doubles per tensor).
 template <typename T, int BITS, int KP, bool STATS = false>
-__global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
+__global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
                                                                      int* __restrict__ error) {
   using Cfg = UmmaCfg<KP>;
   constexpr int NS = Cfg::NS, S = Cfg::STAGES, US = Cfg::USTAGES, ROWB = Cfg::ROWB, NACC = Cfg::NACC, NSUB = Cfg::NSUB;
+  constexpr int kEpiWarps = Cfg::EPI_WARPS, kUmmaThreads = Cfg::THREADS;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   uint8_t* theta_base = smem;                                           // S tiles
@@ -354,6 +382,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       const uint32_t idesc_id = make_idesc(Pack16<T>::kFmt, 16);
       const uint32_t idesc_ug = make_idesc(1, NS);
       const uint64_t desc_id = make_desc(smem_u32(ident), 32);
+      // Descriptors differ only in their start-address field (bits 0-13, address >> 4), so every
+      // operand below is one of these bases plus a small constant.
+      const uint64_t desc_theta0 = make_desc(smem_u32(theta_base), 128);
+      const uint64_t desc_u0 = make_desc(smem_u32(u_base), ROWB);
+      const uint64_t desc_g0 = make_desc(smem_u32(g_base), ROWB);
       int t = 0, rb = 0, item_no = 0;
       bool ok = true;
       for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x, ++item_no) {
@@ -365,30 +398,37 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
         for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128, ++rb) {
           const int u = rb % US;
           if (!mbar_wait<true>(BAR_U_FULL(u), (rb / US) & 1, abort_flag, error, 9)) { ok = false; break; }
-          const uint32_t uhi = smem_u32(u_base + u * 2 * Cfg::U_BYTES), ulo = uhi + Cfg::U_BYTES;
+          const uint64_t desc_uhi = desc_u0 + static_cast<uint64_t>((u * 2 * Cfg::U_BYTES) >> 4);
+          const uint64_t desc_ulo = desc_uhi + static_cast<uint64_t>(Cfg::U_BYTES >> 4);
           for (int sub = 0; sub < nsub; ++sub, ++t) {
             const int s = t % S, b = t % NACC;
             if (!STATS && !mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
             if (t >= NACC && !mbar_wait<true>(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t sbase = smem_u32(theta_base + s * Cfg::THETA_BYTES);
+            const uint64_t desc_theta = desc_theta0 + static_cast<uint64_t>((s * Cfg::THETA_BYTES) >> 4);
             const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
             const int nbox = (min(NS, w.ncols - NS * sub) + 63) / 64;
             // theta -> fp32, 16 columns at a time
-            for (int c = 0; c < nbox && !STATS; ++c)
+            if (!STATS) {
 #pragma unroll
-              for (int k = 0; k < 4; ++k)
-                umma(d + static_cast<uint32_t>(64 * c + 16 * k), make_desc(sbase + c * 16384 + 32 * k, 128), desc_id, idesc_id, 0u);
+              for (int c = 0; c < NS / 64; ++c) {
+                if (c < nbox) {
+#pragma unroll
+                  for (int k = 0; k < 4; ++k)
+                    umma(d + static_cast<uint32_t>(64 * c + 16 * k), desc_theta + static_cast<uint64_t>((c * 16384 + 32 * k) >> 4), desc_id, idesc_id, 0u);
+                }
+              }
+            }
             // + c b U G, split operands
-            const uint64_t desc_ghi = make_desc(smem_u32(g_base + sub * 2 * Cfg::G_BYTES), ROWB);
-            const uint64_t desc_glo = make_desc(smem_u32(g_base + sub * 2 * Cfg::G_BYTES + Cfg::G_BYTES), ROWB);
+            const uint64_t desc_ghi = desc_g0 + static_cast<uint64_t>((sub * 2 * Cfg::G_BYTES) >> 4);
+            const uint64_t desc_glo = desc_ghi + static_cast<uint64_t>(Cfg::G_BYTES >> 4);
 #pragma unroll
             for (int k = 0; k < KP / 16; ++k)
-              umma(d, make_desc(ulo + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, (STATS && k == 0) ? 0u : 1u);
+              umma(d, desc_ulo + static_cast<uint64_t>(2 * k), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, (STATS && k == 0) ? 0u : 1u);
 #pragma unroll
-            for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_glo + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+            for (int k = 0; k < KP / 16; ++k) umma(d, desc_uhi + static_cast<uint64_t>(2 * k), desc_glo + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
 #pragma unroll
-            for (int k = 0; k < KP / 16; ++k) umma(d, make_desc(uhi + 32 * k, ROWB), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+            for (int k = 0; k < KP / 16; ++k) umma(d, desc_uhi + static_cast<uint64_t>(2 * k), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
             umma_commit(BAR_ACC_FULL(b));
           }
           if (ok) umma_commit(BAR_U_FREE(u));   // arrives once every product that reads this U tile has completed
@@ -416,6 +456,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       const TensorDesc& td = p.tensors[w.tensor];
       const uint32_t tid = static_cast<uint32_t>(td.id);
       const int r = td.rank;
+      const uint64_t tcols = static_cast<uint64_t>(td.cols);   // kept in a register: the barriers below force reloads of anything read through td
       // ---- coefficient strips c b G -> K-major hi/lo operands, one per tile of a row block ----
       for (int idx = et; idx < (KP / 2) * (NSUB * NS / 8); idx += kEpiWarps * 32) {
         const int kp = idx / (NSUB * NS / 8), o = idx % (NSUB * NS / 8);
@@ -454,7 +495,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) sweep_umma_kernel(const __gri
       double sum_iso = 0.0, sum_gd = 0.0, sum_z = 0.0;   // STATS only
       for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128) {
         const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
-        const uint64_t row_e = static_cast<uint64_t>(row) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(w.col0 + 32 * cgrp);
+        const uint64_t row_e = static_cast<uint64_t>(row) * tcols + static_cast<uint64_t>(w.col0 + 32 * cgrp);
         for (int sub = 0; sub < nsub; ++sub, ++t) {
           const int s = t % S, b = t % NACC;
           if (!mbar_wait<false>(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
@@ -566,7 +607,7 @@ cudaError_t launch_umma_kp(int kpad, const SweepParams& p, const CUtensorMap* tm
     auto k = sweep_umma_kernel<T, BITS, KPV, STATS>;                                                                 \
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<KPV>::SMEM_BYTES); \
     if (e != cudaSuccess) return e;                                                                                \
-    k<<<grid, kUmmaThreads, UmmaCfg<KPV>::SMEM_BYTES, st>>>(p, tmaps, error);                                      \
+    k<<<grid, UmmaCfg<KPV>::THREADS, UmmaCfg<KPV>::SMEM_BYTES, st>>>(p, tmaps, error);                                      \
   }
   if (kpad == 16) ZGR_LAUNCH_UMMA(16)
   else if (kpad == 32) ZGR_LAUNCH_UMMA(32)
