@@ -200,6 +200,24 @@ def sweep_elements(t: OracleTensor, theta_in: np.ndarray, seed: int, tensor_id: 
     return out
 
 
+def sweep_multi_tensor(t: OracleTensor, seeds: Sequence[int], coeffs: Sequence[float], tensor_id: int, bits: int, a: float, b: float) -> None:
+    """theta <- rnd(theta + sum_q c_q z(seed_q)), in place: the sum over seeds of Algorithm 1
+    ("Recover gradient": sum_t g_t z_t; "Update") applied with a single rounding to the storage type."""
+    acc = decode(t.theta, t.dtype).astype(np.float64).ravel().copy()
+    for seed, c in zip(seeds, coeffs):
+        acc += float(c) * z_tensor(t, seed, tensor_id, bits, a, b).ravel()
+    t.theta[...] = encode(acc, t.dtype).reshape(t.theta.shape)
+
+
+def sweep_multi_elements(t: OracleTensor, theta_in: np.ndarray, seeds: Sequence[int], coeffs: Sequence[float], tensor_id: int, bits: int,
+                         a: float, b: float, idx: np.ndarray) -> np.ndarray:
+    """The same at selected elements; ``theta_in`` holds their current stored values as doubles."""
+    acc = np.ascontiguousarray(theta_in, dtype=np.float64).copy()
+    for seed, c in zip(seeds, coeffs):
+        acc += float(c) * z_elements(t, seed, tensor_id, bits, a, b, idx)
+    return round_to(acc, t.dtype)
+
+
 def stats_tensor(t: OracleTensor, seed: int, tensor_id: int, bits: int, a: float, b: float) -> np.ndarray:
     U, q, sc, ze = t._args()
     out = np.zeros(3, dtype=np.float64)
@@ -251,6 +269,7 @@ class OracleZGR:
         self.a, self.b = mix_scalars(self.alpha, self.d, self.K, self.scale_mode)
         self.active_seed: Optional[int] = None
         self.net = 0.0
+        self.nets = {}                # ledger of the multi-seed calls: seed -> net coefficient applied
 
     def perturb(self, seed: int, c: float) -> None:
         if self.active_seed is not None and self.active_seed != seed:
@@ -263,6 +282,24 @@ class OracleZGR:
     def update_coefficient(self, loss_plus: float, loss_minus: float, lr: float) -> float:
         g = projected_grad(loss_plus, loss_minus, self.eps)
         return -self.net - lr * g
+
+    def sweep_multi(self, seeds: Sequence[int], coeffs: Sequence[float]) -> None:
+        """One pass applying several seeds; the ledger ``self.nets`` records what stays applied per seed."""
+        for l, t in enumerate(self.tensors):
+            sweep_multi_tensor(t, seeds, coeffs, l, self.bits, self.a, self.b)
+        for seed, c in zip(seeds, coeffs):
+            self.nets[seed] = self.nets.get(seed, 0.0) + float(c)
+            if self.nets[seed] == 0.0:
+                del self.nets[seed]
+
+    def restore_update_multi(self, seeds: Sequence[int], loss_plus: Sequence[float], loss_minus: Sequence[float], lr: float):
+        """Eq. (grad) per seed, then theta <- rnd(theta + sum_i (-net_i - lr g_i) z_i) in one pass."""
+        coeffs = [-self.nets.get(s, 0.0) - lr * projected_grad(lp, lm, self.eps) for s, lp, lm in zip(seeds, loss_plus, loss_minus)]
+        for l, t in enumerate(self.tensors):
+            sweep_multi_tensor(t, seeds, coeffs, l, self.bits, self.a, self.b)
+        for s in seeds:
+            self.nets.pop(s, None)
+        return coeffs
 
     def restore_update(self, seed: int, loss_plus: float, loss_minus: float, lr: float) -> float:
         if self.active_seed != seed:
