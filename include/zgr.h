@@ -38,6 +38,7 @@ extern "C" {
 #endif
 
 #define ZGR_MAX_RANK 64 /* largest subspace rank r per tensor */
+#define ZGR_MAX_SEEDS 8 /* most (seed, coefficient) terms one sweep can apply */
 
 enum { ZGR_OK = 0, ZGR_EINVAL = -1, ZGR_ESTATE = -2, ZGR_ECUDA = -3, ZGR_ENOMEM = -4, ZGR_ETOOBIG = -5 };
 
@@ -88,7 +89,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
  * difference": W + eps z_h, then W - eps z_h, reached by scale = +eps followed by scale = -2 eps).
  * The context remembers `seed` and the sum of the scales applied under it.
  * ZGR_EINVAL: scale not finite.  ZGR_ESTATE: a different seed is still active (its
- * restore_update has not been called). */
+ * restore_update has not been called); zgr_sweep_multi is the call that may overlap seeds. */
 int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream);
 
 /* Undo the net perturbation of `seed` and take the projected-gradient step in the same sweep
@@ -97,6 +98,30 @@ int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream);
  * lr = 0 is a pure restore.  Scalars are combined in double on the host and passed to the kernel
  * as fp32.  ZGR_EINVAL: a loss or lr is not finite.  ZGR_ESTATE: `seed` is not the active seed. */
 int zgr_restore_update(zgr_ctx* ctx, uint64_t seed, double loss_plus, double loss_minus, double lr, void* stream);
+
+/* Several seeds in one sweep:  theta_l <- rnd(theta_l + sum_i coeffs[i] * z_l(seeds[i]))  for every tensor,
+ * one rounding.  This is the sum over seeds of Algorithm 1 ("Recover gradient": sum_t g_t z_t, applied
+ * by "Update") as one pass over the weights instead of one pass per seed: the edge server's
+ * aggregation of its clients' projected gradients, a step that averages several perturbation queries,
+ * or the fusion of one query's restore with the next query's perturbation
+ * (seeds = {s_q, s_q+1}, coeffs = {+eps, +eps} after perturb(s_q, +eps), perturb(s_q, -2 eps)).
+ * seeds, coeffs: HOST arrays of n entries, 1 <= n <= ZGR_MAX_SEEDS, seeds pairwise different.
+ * The context adds coeffs[i] to the net coefficient it keeps for seeds[i]; a seed whose net
+ * coefficient returns to exactly 0 is idle again.  Unlike zgr_perturb it may be called while other
+ * seeds are active.  ZGR_EINVAL: null pointer, n out of range, repeated seed, coefficient not finite. */
+int zgr_sweep_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, const double* coeffs, void* stream);
+
+/* zgr_restore_update for n seeds in one sweep (Eq. (grad) per seed; Algorithm 1 "Recover gradient" and
+ * "Update" with the sum over seeds):
+ *     g_i = (loss_plus[i] - loss_minus[i]) / (2 eps),
+ *     theta_l <- rnd(theta_l + sum_i (-net_i - lr g_i) z_l(seeds[i])),
+ * net_i being the net coefficient still applied under seeds[i] (0 for a seed that is not active, which
+ * is the server-side case: nothing to undo, only the update).  `lr` is the step applied per seed: pass
+ * lr/n to average n queries.  The listed seeds are idle afterwards; other active seeds stay active.
+ * All arrays are HOST arrays of n entries, 1 <= n <= ZGR_MAX_SEEDS, seeds pairwise different.
+ * ZGR_EINVAL: null pointer, n out of range, repeated seed, a loss or lr not finite. */
+int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, const double* loss_plus, const double* loss_minus, double lr,
+                             void* stream);
 
 /* Deliver the guided coefficients of one tensor compressed (Sec. 3.4, DTC): from now on
  *     G_l[k][c] = scale[k] * (q[k][c] - zero[k])       (x = lambda (x_quant - delta))
@@ -170,8 +195,9 @@ int zgr_profile_read(zgr_ctx* ctx, zgr_kernel_time* out, int32_t max_entries, in
  * ZGR_ECUDA): the interrupted sweep left the weights partly updated. */
 int zgr_device_status(zgr_ctx* ctx, int32_t* code);
 
-/* Introspection: mixing scalars a, b in double; active seed / net scale (active = 0 when idle);
- * number of kernel launches issued by this context so far. */
+/* Introspection: mixing scalars a, b in double; number of active seeds (0 when idle), the seed most
+ * recently swept and the net coefficient still applied under it; number of kernel launches issued by
+ * this context so far. */
 int zgr_get_scalars(const zgr_ctx* ctx, double* a, double* b);
 int zgr_get_state(const zgr_ctx* ctx, int32_t* active, uint64_t* seed, double* net_scale);
 int64_t zgr_launch_count(const zgr_ctx* ctx);

@@ -273,5 +273,72 @@ __device__ __forceinline__ float coeff1(const TensorDesc& td, const PhiloxKeys& 
                                      static_cast<uint64_t>(k) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(c), unit);
 }
 
+// ---------------------------------------------------------------------------------------------
+// The terms of a sweep.  A sweep applies  sum_q c_q z(seed_q)  with  z = a Z + b U G  (Algorithm 1:
+// one term for a perturbation or a single restore+update; several when the projected gradients of
+// several seeds are applied together, the sum over t in "Recover gradient" / "Update").  MULTI = false
+// reads term[0] with constant addressing, which is the single-seed hot path unchanged.
+// ---------------------------------------------------------------------------------------------
+// sum_q c_q a Z_q  for eight consecutive elements starting at e (a multiple of 8)
+template <int BITS, bool PRECISE, bool MULTI>
+__device__ __forceinline__ void iso8(const SweepParams& p, uint32_t tensor, uint64_t e, float (&z)[8]) {
+  normals8<BITS, PRECISE>(p.term[0].keys, tensor, 0u, e, p.term[0].iso, z);
+  if (MULTI) {
+#pragma unroll 1
+    for (int q = 1; q < p.n_terms; ++q) {
+      float y[8];
+      normals8<BITS, PRECISE>(p.term[q].keys, tensor, 0u, e, p.term[q].iso, y);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) z[i] += y[i];
+    }
+  }
+}
+
+template <int BITS, bool PRECISE, bool MULTI>
+__device__ __forceinline__ float iso1(const SweepParams& p, uint32_t tensor, uint64_t e) {
+  float z = normal1<BITS, PRECISE>(p.term[0].keys, tensor, 0u, e, p.term[0].iso);
+  if (MULTI) {
+#pragma unroll 1
+    for (int q = 1; q < p.n_terms; ++q) z += normal1<BITS, PRECISE>(p.term[q].keys, tensor, 0u, e, p.term[q].iso);
+  }
+  return z;
+}
+
+// sum_q c_q b G_q[k][c .. c+7].  Compressed coefficients do not depend on the seed: they are scaled
+// by the sum of the terms' factors.
+template <int BITS, bool PRECISE, bool MULTI>
+__device__ __forceinline__ void guided8(const TensorDesc& td, const SweepParams& p, int k, int64_t c, float (&g)[8]) {
+  if (!MULTI) {
+    coeffs8<BITS, PRECISE>(td, p.term[0].keys, p.unit, p.term[0].cb, k, c, g);
+  } else if (td.q != nullptr) {
+    float cb = 0.0f;
+    for (int q = 0; q < p.n_terms; ++q) cb += p.term[q].cb;
+    coeffs8<BITS, PRECISE>(td, p.term[0].keys, p.unit, cb, k, c, g);
+  } else {
+    coeffs8<BITS, PRECISE>(td, p.term[0].keys, p.unit, p.term[0].cb, k, c, g);
+#pragma unroll 1
+    for (int q = 1; q < p.n_terms; ++q) {
+      float y[8];
+      coeffs8<BITS, PRECISE>(td, p.term[q].keys, p.unit, p.term[q].cb, k, c, y);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) g[i] += y[i];
+    }
+  }
+}
+
+template <int BITS, bool PRECISE, bool MULTI>
+__device__ __forceinline__ float guided1(const TensorDesc& td, const SweepParams& p, int k, int64_t c) {
+  if (!MULTI) return coeff1<BITS, PRECISE>(td, p.term[0].keys, p.unit, p.term[0].cb, k, c);
+  if (td.q != nullptr) {
+    float cb = 0.0f;
+    for (int q = 0; q < p.n_terms; ++q) cb += p.term[q].cb;
+    return coeff1<BITS, PRECISE>(td, p.term[0].keys, p.unit, cb, k, c);
+  }
+  float g = 0.0f;
+#pragma unroll 1
+  for (int q = 0; q < p.n_terms; ++q) g += coeff1<BITS, PRECISE>(td, p.term[q].keys, p.unit, p.term[q].cb, k, c);
+  return g;
+}
+
 }  // namespace zgr
 #endif  // ZGR_DEVICE_CUH_

@@ -48,9 +48,10 @@ struct zgr_ctx {
   bool stats_planned = false;
   WorkItem* d_stats_items = nullptr;
   double* d_stats = nullptr;
-  bool active = false;
-  uint64_t seed = 0;
-  double net = 0;
+  std::map<uint64_t, double> ledger;  // seeds whose perturbation is applied to the weights -> sum of the coefficients applied
+  uint64_t last_seed = 0;             // most recently swept seed (introspection)
+  std::vector<Group> groups_multi;    // plan of multi-seed sweeps when it differs from `groups` (legacy tensor-core path only)
+  bool multi_planned = false;
   int sticky = 0;                     // first CUDA failure, returned by every later call
   int64_t launches = 0;
   bool profiling = false;
@@ -136,7 +137,7 @@ int blocks_per_sm(int path) {
 // an exact fp32 contraction); `kernel_dtype` >= 0 overrides only the type the kernel reads and writes,
 // which lets the test hook run a 16-bit tensor's kernel family on an fp32 image.
 void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, bool guided_on, int bits, int sm_count,
-          std::vector<Group>& out, int kernel_dtype = -1) {
+          std::vector<Group>& out, int kernel_dtype = -1, bool multi = false) {
   int64_t total = 0;
   for (int l : which) total += descs[l].rows * descs[l].cols;
   // elements per item: enough items for ~16 rounds over the resident CTAs, but large enough that the
@@ -174,11 +175,13 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
     }
     const bool vec = aligned && (t.cols % 8 == 0);
     int path, kpad, strip, row_step;
-    if (!vec || (t.rank > 8 && t.Ufrag == nullptr)) {
+    const bool umma_ok = t.umma && kernel_dtype < 0;
+    if (!vec || (t.rank > 8 && t.Ufrag == nullptr) || (multi && t.rank > 8 && !umma_ok)) {
+      // (the legacy tensor-core kernel applies one term per sweep; several terms take the fallback)
       path = PATH_GENERIC; kpad = 0; strip = 64; row_step = 1;
     } else if (t.rank <= 8) {
       path = PATH_FMA; kpad = t.rank <= 4 ? 4 : 8; strip = 256; row_step = 1;
-    } else if (t.umma && kernel_dtype < 0) {
+    } else if (umma_ok) {
       path = PATH_UMMA; kpad = t.kpad; strip = umma_strip_cols(kpad); row_step = 128;
     } else {
       path = PATH_MMA; kpad = t.rank <= 16 ? 16 : (t.rank <= 32 ? 32 : 64);
@@ -232,14 +235,18 @@ int upload_groups(zgr_ctx* ctx, std::vector<Group>& groups) {
   return ZGR_OK;
 }
 
-// One sweep  theta <- rnd(theta + c z(seed))  over the planned groups.
-int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, uint64_t seed, double c, cudaStream_t st) {
+// One sweep  theta <- rnd(theta + sum_q c_q z(seed_q))  over the planned groups (n terms, 1 <= n <= kMaxTerms).
+int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, int n, const uint64_t* seeds, const double* c, cudaStream_t st) {
   SweepParams p;
-  p.keys = make_keys(seed);
-  p.iso = make_scale(c * ctx->a, ctx->cfg.bits_per_normal);
+  std::memset(&p, 0, sizeof(p));
+  for (int q = 0; q < n; ++q) {
+    p.term[q].keys = make_keys(seeds[q]);
+    p.term[q].iso = make_scale(c[q] * ctx->a, ctx->cfg.bits_per_normal);
+    p.term[q].cb = static_cast<float>(c[q] * ctx->b);
+  }
+  p.n_terms = n;
   p.unit = make_scale(1.0, ctx->cfg.bits_per_normal);
   p.tensors = d_descs;
-  p.cb = static_cast<float>(c * ctx->b);
   p.stats = nullptr;
   for (Group& g : groups) {
     if (g.items.empty()) continue;
@@ -270,6 +277,31 @@ int flush_descs(zgr_ctx* ctx, cudaStream_t st) {
 }
 
 bool is_finite(double x) { return std::isfinite(x); }
+
+// Book-keeping of the coefficients applied under each seed; a seed whose coefficients cancel is idle again.
+void ledger_add(zgr_ctx* ctx, uint64_t seed, double c) {
+  double& net = ctx->ledger[seed];
+  net += c;
+  if (net == 0.0) ctx->ledger.erase(seed);
+  ctx->last_seed = seed;
+}
+
+// Plan used by sweeps with several terms: the sweep plan itself unless it contains the legacy
+// tensor-core kernel, which applies one term per sweep; those tensors are re-planned onto the fallback.
+std::vector<Group>& multi_groups(zgr_ctx* ctx, int* rc) {
+  *rc = ZGR_OK;
+  bool legacy = false;
+  for (const Group& g : ctx->groups) legacy = legacy || (g.kc.path == PATH_MMA && !g.items.empty());
+  if (!legacy) return ctx->groups;
+  if (!ctx->multi_planned) {
+    std::vector<int> all(ctx->descs.size());
+    for (size_t l = 0; l < all.size(); ++l) all[l] = static_cast<int>(l);
+    plan(ctx->descs, all, ctx->b != 0.0, ctx->cfg.bits_per_normal, ctx->sm_count, ctx->groups_multi, -1, true);
+    *rc = upload_groups(ctx, ctx->groups_multi);
+    ctx->multi_planned = true;
+  }
+  return ctx->groups_multi;
+}
 
 }  // namespace
 
@@ -410,33 +442,78 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
 int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream) {
   if (!ctx || !is_finite(scale)) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
-  if (ctx->active && ctx->seed != seed) return ZGR_ESTATE;
+  if (!ctx->ledger.empty() && !(ctx->ledger.size() == 1 && ctx->ledger.count(seed) == 1)) return ZGR_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
-  rc = sweep(ctx, ctx->groups, ctx->d_descs, seed, scale, st);
+  rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, st);
   if (rc != ZGR_OK) return rc;
-  ctx->active = true;
-  ctx->seed = seed;
-  ctx->net += scale;
+  ledger_add(ctx, seed, scale);
   return ZGR_OK;
 }
 
 int zgr_restore_update(zgr_ctx* ctx, uint64_t seed, double loss_plus, double loss_minus, double lr, void* stream) {
   if (!ctx || !is_finite(loss_plus) || !is_finite(loss_minus) || !is_finite(lr)) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
-  if (!ctx->active || ctx->seed != seed) return ZGR_ESTATE;
+  const auto active = ctx->ledger.find(seed);
+  if (active == ctx->ledger.end()) return ZGR_ESTATE;
   // Eq. (grad): projected gradient; Algorithm 1 "Update": W <- W - eta g z, fused with the restore
   const double g = (loss_plus - loss_minus) / (2.0 * ctx->cfg.eps);
-  const double c = -ctx->net - lr * g;
+  const double c = -active->second - lr * g;
   if (!is_finite(c)) return ZGR_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
-  rc = sweep(ctx, ctx->groups, ctx->d_descs, seed, c, st);
+  rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &c, st);
   if (rc != ZGR_OK) return rc;
-  ctx->active = false;
-  ctx->net = 0.0;
+  ctx->ledger.erase(seed);
+  ctx->last_seed = seed;
+  return ZGR_OK;
+}
+
+int zgr_sweep_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, const double* coeffs, void* stream) {
+  if (!ctx || !seeds || !coeffs || n < 1 || n > ZGR_MAX_SEEDS) return ZGR_EINVAL;
+  for (int32_t i = 0; i < n; ++i) {
+    if (!is_finite(coeffs[i])) return ZGR_EINVAL;
+    for (int32_t j = 0; j < i; ++j)
+      if (seeds[j] == seeds[i]) return ZGR_EINVAL;
+  }
+  if (ctx->sticky) return ctx->sticky;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = flush_descs(ctx, st);
+  if (rc != ZGR_OK) return rc;
+  std::vector<Group>& groups = n > 1 ? multi_groups(ctx, &rc) : ctx->groups;
+  if (rc != ZGR_OK) return rc;
+  rc = sweep(ctx, groups, ctx->d_descs, n, seeds, coeffs, st);
+  if (rc != ZGR_OK) return rc;
+  for (int32_t i = 0; i < n; ++i) ledger_add(ctx, seeds[i], coeffs[i]);
+  return ZGR_OK;
+}
+
+int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, const double* loss_plus, const double* loss_minus, double lr,
+                             void* stream) {
+  if (!ctx || !seeds || !loss_plus || !loss_minus || n < 1 || n > ZGR_MAX_SEEDS || !is_finite(lr)) return ZGR_EINVAL;
+  double c[ZGR_MAX_SEEDS];
+  for (int32_t i = 0; i < n; ++i) {
+    if (!is_finite(loss_plus[i]) || !is_finite(loss_minus[i])) return ZGR_EINVAL;
+    for (int32_t j = 0; j < i; ++j)
+      if (seeds[j] == seeds[i]) return ZGR_EINVAL;
+    // Eq. (grad) per seed; Algorithm 1 "Recover gradient" sums g_t z_t over the seeds, "Update" applies it
+    const double g = (loss_plus[i] - loss_minus[i]) / (2.0 * ctx->cfg.eps);
+    const auto it = ctx->ledger.find(seeds[i]);
+    c[i] = -(it == ctx->ledger.end() ? 0.0 : it->second) - lr * g;
+    if (!is_finite(c[i])) return ZGR_EINVAL;
+  }
+  if (ctx->sticky) return ctx->sticky;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = flush_descs(ctx, st);
+  if (rc != ZGR_OK) return rc;
+  std::vector<Group>& groups = n > 1 ? multi_groups(ctx, &rc) : ctx->groups;
+  if (rc != ZGR_OK) return rc;
+  rc = sweep(ctx, groups, ctx->d_descs, n, seeds, c, st);
+  if (rc != ZGR_OK) return rc;
+  for (int32_t i = 0; i < n; ++i) ctx->ledger.erase(seeds[i]);
+  ctx->last_seed = seeds[n - 1];
   return ZGR_OK;
 }
 
@@ -445,7 +522,7 @@ int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const floa
   if (!q || !scale || bits != 8) return ZGR_EINVAL;
   TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
   if (td.rank == 0) return ZGR_EINVAL;
-  if (ctx->active) return ZGR_ESTATE;
+  if (!ctx->ledger.empty()) return ZGR_ESTATE;
   td.q = q;
   td.qscale = scale;
   td.qzero = zero;
@@ -457,7 +534,7 @@ int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor) {
   if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
   TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
   if (td.rank == 0) return ZGR_EINVAL;
-  if (ctx->active) return ZGR_ESTATE;
+  if (!ctx->ledger.empty()) return ZGR_ESTATE;
   td.q = nullptr;
   td.qscale = nullptr;
   td.qzero = nullptr;
@@ -497,13 +574,15 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
   rc = check(ctx, cudaMemsetAsync(ctx->d_stats, 0, 3 * n * sizeof(double), st));
   if (rc != ZGR_OK) return rc;
   SweepParams p;
-  p.keys = make_keys(seed);
-  p.iso = make_scale(ctx->a, ctx->cfg.bits_per_normal);
+  std::memset(&p, 0, sizeof(p));
+  p.n_terms = 1;
+  p.term[0].keys = make_keys(seed);
+  p.term[0].iso = make_scale(ctx->a, ctx->cfg.bits_per_normal);
   p.unit = make_scale(1.0, ctx->cfg.bits_per_normal);
   p.tensors = ctx->d_descs;
   p.items = ctx->d_stats_items;
   p.n_items = static_cast<int32_t>(ctx->stats_items.size());
-  p.cb = static_cast<float>(ctx->b);
+  p.term[0].cb = static_cast<float>(ctx->b);
   p.stats = ctx->d_stats;
   if (p.n_items > 0) {
     const int grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * 4));
@@ -553,7 +632,8 @@ int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, voi
   if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(d_one, one.data(), sizeof(TensorDesc), cudaMemcpyHostToDevice));
   if (rc == ZGR_OK) rc = upload_groups(ctx, groups);
   if (rc == ZGR_OK) rc = check(ctx, cudaMemsetAsync(dev_out, 0, static_cast<size_t>(one[0].rows * one[0].cols) * sizeof(float), st));
-  if (rc == ZGR_OK) rc = sweep(ctx, groups, d_one, seed, 1.0, st);
+  const double one_scale = 1.0;
+  if (rc == ZGR_OK) rc = sweep(ctx, groups, d_one, 1, &seed, &one_scale, st);
   if (rc == ZGR_OK) rc = check(ctx, cudaStreamSynchronize(st));
   for (size_t i = owned_before; i < ctx->owned.size(); ++i) cudaFree(ctx->owned[i]);
   ctx->owned.resize(owned_before);
@@ -565,7 +645,7 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
   TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
   if (td.rank == 0) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
-  if (ctx->active) return ZGR_ESTATE;
+  if (!ctx->ledger.empty()) return ZGR_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = ZGR_OK;
   if (U_src != nullptr && U_src != td.U) {
@@ -597,7 +677,8 @@ int zgr_profile_read(zgr_ctx* ctx, zgr_kernel_time* out, int32_t max_entries, in
   const int rc = check(ctx, cudaDeviceSynchronize());
   if (rc != ZGR_OK) return rc;
   int32_t n = 0;
-  for (Group& g : ctx->groups) {
+  for (std::vector<Group>* gs : {&ctx->groups, &ctx->groups_multi})
+  for (Group& g : *gs) {
     if (g.timed.empty()) continue;
     double total = 0.0;
     for (auto& ev : g.timed) {
@@ -644,9 +725,10 @@ int zgr_get_scalars(const zgr_ctx* ctx, double* a, double* b) {
 
 int zgr_get_state(const zgr_ctx* ctx, int32_t* active, uint64_t* seed, double* net_scale) {
   if (!ctx || !active || !seed || !net_scale) return ZGR_EINVAL;
-  *active = ctx->active ? 1 : 0;
-  *seed = ctx->seed;
-  *net_scale = ctx->net;
+  *active = static_cast<int32_t>(ctx->ledger.size());
+  const auto it = ctx->ledger.find(ctx->last_seed);
+  *seed = ctx->last_seed;
+  *net_scale = it == ctx->ledger.end() ? 0.0 : it->second;
   return ZGR_OK;
 }
 
@@ -654,11 +736,12 @@ int64_t zgr_launch_count(const zgr_ctx* ctx) { return ctx ? ctx->launches : -1; 
 
 void zgr_destroy(zgr_ctx* ctx) {
   if (!ctx) return;
-  for (Group& g : ctx->groups)
-    for (auto& ev : g.timed) {
-      cudaEventDestroy(ev.first);
-      cudaEventDestroy(ev.second);
-    }
+  for (std::vector<Group>* gs : {&ctx->groups, &ctx->groups_multi})
+    for (Group& g : *gs)
+      for (auto& ev : g.timed) {
+        cudaEventDestroy(ev.first);
+        cudaEventDestroy(ev.second);
+      }
   for (void* p : ctx->owned) cudaFree(p);
   delete ctx;
 }

@@ -50,15 +50,25 @@ struct NormalScale {
   float u1_off;   // 2^-(nb+1) - 1
 };
 
-// Per-launch constants (passed by value in the kernel parameter space).
+// One (seed, coefficient) term of a sweep  theta <- rnd(theta + sum_q c_q z(seed_q)).
+struct SeedTerm {
+  PhiloxKeys keys;       // round keys of seed_q
+  NormalScale iso;       // isotropic normals of this seed, scaled by c_q * a
+  float cb;              // c_q * b : coefficient of U G(seed_q)
+};
+
+constexpr int kMaxTerms = 8;   // ZGR_MAX_SEEDS of the C ABI
+
+// Per-launch constants (passed by value in the kernel parameter space).  A single-seed sweep uses
+// term[0] only, addressed with a compile-time index so that its round keys stay constant-bank
+// operands; multi-seed instantiations loop over term[0 .. n_terms).
 struct SweepParams {
-  PhiloxKeys keys;
-  NormalScale iso;       // isotropic normals, scaled by c*a
+  SeedTerm term[kMaxTerms];
+  int32_t n_terms;
   NormalScale unit;      // coefficient normals, unscaled
   const TensorDesc* tensors;
   const WorkItem* items;
   int32_t n_items;
-  float cb;              // c * b : coefficient of U G
   double* stats;         // 3 doubles per tensor (stats kernels only)
 };
 

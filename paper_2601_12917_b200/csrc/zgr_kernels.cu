@@ -29,7 +29,7 @@ constexpr int kWarps = kThreads / 32;
 // ---------------------------------------------------------------------------------------------
 // isotropic sweep
 // ---------------------------------------------------------------------------------------------
-template <typename T, int BITS, bool PRECISE>
+template <typename T, int BITS, bool PRECISE, bool MULTI>
 __global__ void __launch_bounds__(kThreads) sweep_iso_kernel(const __grid_constant__ SweepParams p) {
   for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
     const WorkItem w = p.items[it];
@@ -43,13 +43,13 @@ __global__ void __launch_bounds__(kThreads) sweep_iso_kernel(const __grid_consta
       const int64_t e = e0 + 8 * v;
       float th[8], z[8];
       Storage<T>::load8(base + e, th);
-      normals8<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso, z);
+      iso8<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e), z);
 #pragma unroll
       for (int i = 0; i < 8; ++i) th[i] += z[i];
       Storage<T>::store8(base + e, th);
     }
     for (int64_t e = e0 + 8 * n_oct + threadIdx.x; e < e0 + count; e += kThreads) {
-      const float z = normal1<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso);
+      const float z = iso1<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e));
       Storage<T>::store1(base + e, Storage<T>::load1(base + e) + z);
     }
   }
@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kThreads) sweep_iso_kernel(const __grid_consta
 // [8l, 8l+8) of the strip and keeps its R x 8 coefficients in registers; the eight warps walk
 // the rows of the item in an interleaved fashion, each row being one 128-bit access per lane.
 // ---------------------------------------------------------------------------------------------
-template <typename T, int BITS, bool PRECISE, int R>
+template <typename T, int BITS, bool PRECISE, int R, bool MULTI>
 __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_constant__ SweepParams p) {
   __shared__ float Gs[R][256 + 8];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_con
       if (8 * o < w.ncols) {
         float g[8];
         if (k < r) {
-          coeffs8<BITS, PRECISE>(td, p.keys, p.unit, p.cb, k, w.col0 + 8 * o, g);
+          guided8<BITS, PRECISE, MULTI>(td, p, k, w.col0 + 8 * o, g);
         } else {
 #pragma unroll
           for (int i = 0; i < 8; ++i) g[i] = 0.0f;
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_con
         const int64_t e = row * cols + w.col0 + 8 * lane;
         float th[8], z[8];
         Storage<T>::load8(base + e, th);
-        normals8<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso, z);
+        iso8<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e), z);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           float acc = z[i];  // the perturbation is summed on its own scale, then added to theta once
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_con
 // ---------------------------------------------------------------------------------------------
 // any shape: one element per thread, strip of 64 columns, rank <= 64.
 // ---------------------------------------------------------------------------------------------
-template <typename T, int BITS, bool PRECISE>
+template <typename T, int BITS, bool PRECISE, bool MULTI>
 __global__ void __launch_bounds__(kThreads) sweep_generic_kernel(const __grid_constant__ SweepParams p) {
   __shared__ float Gs[64][64 + 1];
   const int cl = threadIdx.x & 63, rg = threadIdx.x >> 6;
@@ -142,14 +142,14 @@ __global__ void __launch_bounds__(kThreads) sweep_generic_kernel(const __grid_co
     __syncthreads();
     for (int idx = threadIdx.x; idx < r * 64; idx += kThreads) {
       const int k = idx >> 6, c = idx & 63;
-      if (c < w.ncols) Gs[k][c] = coeff1<BITS, PRECISE>(td, p.keys, p.unit, p.cb, k, w.col0 + c);
+      if (c < w.ncols) Gs[k][c] = guided1<BITS, PRECISE, MULTI>(td, p, k, w.col0 + c);
     }
     __syncthreads();
     if (cl >= w.ncols) continue;
     const int64_t row_end = w.row0_or_e0 + w.nrows_or_count;
     for (int64_t row = w.row0_or_e0 + rg; row < row_end; row += kThreads / 64) {
       const int64_t e = row * td.cols + w.col0 + cl;
-      float acc = normal1<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso);
+      float acc = iso1<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e));
       for (int k = 0; k < r; ++k) acc = fmaf(__ldg(td.U + row * r + k), Gs[k][cl], acc);
       Storage<T>::store1(base + e, Storage<T>::load1(base + e) + acc);
     }
@@ -241,13 +241,13 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_mma_kernel(const __grid_con
       const int c = 8 * o;
       float g0[8], g1[8];
       if (c < w.ncols && 2 * kp < r) {
-        coeffs8<BITS, PRECISE>(td, p.keys, p.unit, p.cb, 2 * kp, w.col0 + c, g0);
+        guided8<BITS, PRECISE, false>(td, p, 2 * kp, w.col0 + c, g0);
       } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) g0[i] = 0.0f;
       }
       if (c < w.ncols && 2 * kp + 1 < r) {
-        coeffs8<BITS, PRECISE>(td, p.keys, p.unit, p.cb, 2 * kp + 1, w.col0 + c, g1);
+        guided8<BITS, PRECISE, false>(td, p, 2 * kp + 1, w.col0 + c, g1);
       } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) g1[i] = 0.0f;
@@ -323,7 +323,7 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_mma_kernel(const __grid_con
           if (rok && (hf ? act1 : act0)) {
             const int64_t e = rows2[h] * cols + colw + 32 * hf + 8 * t;
             float z[8], th[8];
-            normals8<BITS, PRECISE>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso, z);
+            iso8<BITS, PRECISE, false>(p, tid, static_cast<uint64_t>(e), z);
 #pragma unroll
             for (int i = 0; i < 8; ++i) th[i] = acc[4 * hf + (i >> 1)][2 * h + (i & 1)] + z[i];
             Storage<T>::store8(base + e, th);
@@ -346,11 +346,11 @@ __global__ void __launch_bounds__(kThreads) stats_kernel(const __grid_constant__
     const WorkItem w = p.items[it];
     const TensorDesc& td = p.tensors[w.tensor];
     const uint32_t tid = static_cast<uint32_t>(td.id);
-    const int r = p.cb != 0.0f ? td.rank : 0;
+    const int r = p.term[0].cb != 0.0f ? td.rank : 0;
     __syncthreads();
     for (int idx = threadIdx.x; idx < r * 64; idx += kThreads) {
       const int k = idx >> 6, c = idx & 63;
-      if (c < w.ncols) Gs[k][c] = coeff1<BITS, true>(td, p.keys, p.unit, p.cb, k, w.col0 + c);
+      if (c < w.ncols) Gs[k][c] = guided1<BITS, true, false>(td, p, k, w.col0 + c);
     }
     __syncthreads();
     double s0 = 0.0, s1 = 0.0, s2 = 0.0;
@@ -358,7 +358,7 @@ __global__ void __launch_bounds__(kThreads) stats_kernel(const __grid_constant__
       const int64_t row_end = w.row0_or_e0 + w.nrows_or_count;
       for (int64_t row = w.row0_or_e0 + rg; row < row_end; row += kThreads / 64) {
         const int64_t e = row * td.cols + w.col0 + cl;
-        const float iso = normal1<BITS, true>(p.keys, tid, 0u, static_cast<uint64_t>(e), p.iso);
+        const float iso = iso1<BITS, true, false>(p, tid, static_cast<uint64_t>(e));
         float gd = 0.0f;
         for (int k = 0; k < r; ++k) gd = fmaf(__ldg(td.U + row * td.rank + k), Gs[k][cl], gd);
         s0 += static_cast<double>(iso) * iso;
@@ -420,22 +420,22 @@ __global__ void philox_blocks_kernel(PhiloxKeys keys, uint32_t tensor, uint32_t 
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-template <typename T, int BITS, bool PRECISE>
+template <typename T, int BITS, bool PRECISE, bool MULTI>
 cudaError_t launch_typed(const KernelChoice& kc, const SweepParams& p, int grid, cudaStream_t st) {
   switch (kc.path) {
     case PATH_ISO:
-      sweep_iso_kernel<T, BITS, PRECISE><<<grid, kThreads, 0, st>>>(p);
+      sweep_iso_kernel<T, BITS, PRECISE, MULTI><<<grid, kThreads, 0, st>>>(p);
       break;
     case PATH_FMA:
-      if (kc.kpad == 4) sweep_fma_kernel<T, BITS, PRECISE, 4><<<grid, kThreads, 0, st>>>(p);
-      else sweep_fma_kernel<T, BITS, PRECISE, 8><<<grid, kThreads, 0, st>>>(p);
+      if (kc.kpad == 4) sweep_fma_kernel<T, BITS, PRECISE, 4, MULTI><<<grid, kThreads, 0, st>>>(p);
+      else sweep_fma_kernel<T, BITS, PRECISE, 8, MULTI><<<grid, kThreads, 0, st>>>(p);
       break;
     case PATH_GENERIC:
-      sweep_generic_kernel<T, BITS, PRECISE><<<grid, kThreads, 0, st>>>(p);
+      sweep_generic_kernel<T, BITS, PRECISE, MULTI><<<grid, kThreads, 0, st>>>(p);
       break;
     case PATH_MMA: {
-      if constexpr (PRECISE) {
-        return cudaErrorInvalidValue;  // the split-bf16 contraction cannot meet the fp32 tolerance
+      if constexpr (PRECISE || MULTI) {
+        return cudaErrorInvalidValue;  // the split-bf16 contraction cannot meet the fp32 tolerance; several terms go through the tcgen05 or the fallback kernel
       } else {
         const size_t smem = mma_smem_bytes(kc.kpad);
         if (kc.kpad == 16) {
@@ -460,18 +460,18 @@ cudaError_t launch_typed(const KernelChoice& kc, const SweepParams& p, int grid,
   return cudaGetLastError();
 }
 
-template <typename T>
+template <typename T, bool MULTI>
 cudaError_t launch_dtype(const KernelChoice& kc, const SweepParams& p, int grid, cudaStream_t st) {
   if (kc.precise) {
     if constexpr (sizeof(T) == 4) {
-      if (kc.bits == 32) return launch_typed<T, 32, true>(kc, p, grid, st);
-      return launch_typed<T, 16, true>(kc, p, grid, st);
+      if (kc.bits == 32) return launch_typed<T, 32, true, MULTI>(kc, p, grid, st);
+      return launch_typed<T, 16, true, MULTI>(kc, p, grid, st);
     } else {
       return cudaErrorInvalidValue;  // 16-bit storage never needs the accurate transform
     }
   }
-  if (kc.bits == 32) return launch_typed<T, 32, false>(kc, p, grid, st);
-  return launch_typed<T, 16, false>(kc, p, grid, st);
+  if (kc.bits == 32) return launch_typed<T, 32, false, MULTI>(kc, p, grid, st);
+  return launch_typed<T, 16, false, MULTI>(kc, p, grid, st);
 }
 
 }  // namespace
@@ -481,10 +481,18 @@ int mma_rows_per_iter(int kpad) { return kpad == 64 ? 32 : 16; }
 size_t mma_smem_bytes(int kpad) { return static_cast<size_t>(mma_strip_cols(kpad)) * kpad * 2 * 2; }
 
 cudaError_t launch_sweep(const KernelChoice& kc, const SweepParams& p, int grid, cudaStream_t st) {
+  if (p.n_terms > 1) {
+    switch (kc.dtype) {
+      case 0: return launch_dtype<float, true>(kc, p, grid, st);
+      case 1: return launch_dtype<__half, true>(kc, p, grid, st);
+      case 2: return launch_dtype<__nv_bfloat16, true>(kc, p, grid, st);
+      default: return cudaErrorInvalidValue;
+    }
+  }
   switch (kc.dtype) {
-    case 0: return launch_dtype<float>(kc, p, grid, st);
-    case 1: return launch_dtype<__half>(kc, p, grid, st);
-    case 2: return launch_dtype<__nv_bfloat16>(kc, p, grid, st);
+    case 0: return launch_dtype<float, false>(kc, p, grid, st);
+    case 1: return launch_dtype<__half, false>(kc, p, grid, st);
+    case 2: return launch_dtype<__nv_bfloat16, false>(kc, p, grid, st);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -265,8 +265,11 @@ struct TileCoord {
 // that a CTA touches up to 256*NSUB contiguous bytes of every row and loads each U tile once.
 // STATS = true turns the same pipeline into the norm bookkeeping: no weights are loaded or stored,
 // D = b U G only, and the epilogue accumulates sum (a Z)^2, sum (b U G)^2 and sum z^2 per tensor
-// (p.iso carries the scale a, p.cb = b, p.stats the three doubles per tensor).
-template <typename T, int BITS, int KP, bool STATS = false>
+// (term[0].iso carries the scale a, term[0].cb = b, p.stats the three doubles per tensor).
+// MULTI = true applies several (seed, coefficient) terms in the one pass: the coefficient strips of
+// the terms are summed before the split (U (sum_q c_q b G_q) is one product), the isotropic normals
+// are added term by term in the epilogue.
+template <typename T, int BITS, int KP, bool STATS = false, bool MULTI = false>
 __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
                                                                      int* __restrict__ error) {
   using Cfg = UmmaCfg<KP>;
@@ -479,13 +482,13 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
         if (cc >= ((w.ncols + NS - 1) / NS) * NS) continue;   // tiles of this item that do not exist
         float g0[8], g1[8];
         if (cc < w.ncols && 2 * kp < r) {
-          coeffs8<BITS, false>(td, p.keys, p.unit, p.cb, 2 * kp, w.col0 + cc, g0);
+          guided8<BITS, false, MULTI>(td, p, 2 * kp, w.col0 + cc, g0);
         } else {
 #pragma unroll
           for (int i = 0; i < 8; ++i) g0[i] = 0.0f;
         }
         if (cc < w.ncols && 2 * kp + 1 < r) {
-          coeffs8<BITS, false>(td, p.keys, p.unit, p.cb, 2 * kp + 1, w.col0 + cc, g1);
+          guided8<BITS, false, MULTI>(td, p, 2 * kp + 1, w.col0 + cc, g1);
         } else {
 #pragma unroll
           for (int i = 0; i < 8; ++i) g1[i] = 0.0f;
@@ -536,7 +539,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
 #pragma unroll
                 for (int i = 0; i < 8; ++i) zi[i] = 0.0f;
                 const uint32_t lo = oct0_lo + static_cast<uint32_t>(o);
-                normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, zi);
+                normals8_acc<BITS>(p.term[0].keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.term[0].iso, zi);
                 const bool live = row < row_end && NS * sub + 32 * cgrp + 8 * o < w.ncols;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
@@ -559,7 +562,12 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
 #pragma unroll
               for (int i = 0; i < 8; ++i) acc[i] = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
               const uint32_t lo = oct0_lo + static_cast<uint32_t>(o);
-              normals8_acc<BITS>(p.keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.iso, acc);
+              normals8_acc<BITS>(p.term[0].keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.term[0].iso, acc);
+              if (MULTI) {
+#pragma unroll 1
+                for (int q = 1; q < p.n_terms; ++q)
+                  normals8_acc<BITS>(p.term[q].keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.term[q].iso, acc);
+              }
               const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
                                          Pack16<T>::pack(acc[6], acc[7]));
               sts128(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4), q);
@@ -620,11 +628,11 @@ size_t umma_smem_bytes(int kpad) {
 int umma_strip_cols(int kpad) { return kpad == 64 ? UmmaCfg<64>::NS * UmmaCfg<64>::NSUB : (kpad == 32 ? UmmaCfg<32>::NS * UmmaCfg<32>::NSUB : UmmaCfg<16>::NS * UmmaCfg<16>::NSUB); }
 
 namespace {
-template <typename T, int BITS, bool STATS = false>
+template <typename T, int BITS, bool STATS = false, bool MULTI = false>
 cudaError_t launch_umma_kp(int kpad, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
 #define ZGR_LAUNCH_UMMA(KPV)                                                                                       \
   {                                                                                                                \
-    auto k = sweep_umma_kernel<T, BITS, KPV, STATS>;                                                                 \
+    auto k = sweep_umma_kernel<T, BITS, KPV, STATS, MULTI>;                                                               \
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<KPV>::SMEM_BYTES); \
     if (e != cudaSuccess) return e;                                                                                \
     k<<<grid, UmmaCfg<KPV>::THREADS, UmmaCfg<KPV>::SMEM_BYTES, st>>>(p, tmaps, error);                                      \
@@ -637,14 +645,20 @@ cudaError_t launch_umma_kp(int kpad, const SweepParams& p, const CUtensorMap* tm
 }
 }  // namespace
 
+namespace {
+template <typename T>
+cudaError_t launch_umma_typed(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
+  if (p.n_terms > 1) {
+    return kc.bits == 32 ? launch_umma_kp<T, 32, false, true>(kc.kpad, p, tmaps, error, grid, st)
+                         : launch_umma_kp<T, 16, false, true>(kc.kpad, p, tmaps, error, grid, st);
+  }
+  return kc.bits == 32 ? launch_umma_kp<T, 32>(kc.kpad, p, tmaps, error, grid, st) : launch_umma_kp<T, 16>(kc.kpad, p, tmaps, error, grid, st);
+}
+}  // namespace
+
 cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
-  if (kc.dtype == 2) {
-    return kc.bits == 32 ? launch_umma_kp<__nv_bfloat16, 32>(kc.kpad, p, tmaps, error, grid, st)
-                         : launch_umma_kp<__nv_bfloat16, 16>(kc.kpad, p, tmaps, error, grid, st);
-  }
-  if (kc.dtype == 1) {
-    return kc.bits == 32 ? launch_umma_kp<__half, 32>(kc.kpad, p, tmaps, error, grid, st) : launch_umma_kp<__half, 16>(kc.kpad, p, tmaps, error, grid, st);
-  }
+  if (kc.dtype == 2) return launch_umma_typed<__nv_bfloat16>(kc, p, tmaps, error, grid, st);
+  if (kc.dtype == 1) return launch_umma_typed<__half>(kc, p, tmaps, error, grid, st);
   return cudaErrorInvalidValue;
 }
 

@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.zgr_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(ZgrTensor), i32, ctypes.POINTER(ZgrConfig)]
         L.zgr_perturb.argtypes = [vp, u64, dbl, vp]
         L.zgr_restore_update.argtypes = [vp, u64, dbl, dbl, dbl, vp]
+        L.zgr_sweep_multi.argtypes = [vp, i32, ctypes.POINTER(u64), ctypes.POINTER(dbl), vp]
+        L.zgr_restore_update_multi.argtypes = [vp, i32, ctypes.POINTER(u64), ctypes.POINTER(dbl), ctypes.POINTER(dbl), dbl, vp]
         L.zgr_set_coeffs_dtc.argtypes = [vp, i32, vp, vp, vp, i32]
         L.zgr_clear_coeffs.argtypes = [vp, i32]
         L.zgr_get_stats.argtypes = [vp, u64, ctypes.POINTER(dbl), vp]
@@ -82,7 +84,7 @@ def lib() -> ctypes.CDLL:
         L.zgr_strerror.restype = ctypes.c_char_p
         for name in ("zgr_init", "zgr_perturb", "zgr_restore_update", "zgr_set_coeffs_dtc", "zgr_clear_coeffs", "zgr_get_stats",
                      "zgr_debug_philox", "zgr_debug_z", "zgr_get_scalars", "zgr_get_state", "zgr_update_subspace", "zgr_profile",
-                     "zgr_profile_read"):
+                     "zgr_profile_read", "zgr_sweep_multi", "zgr_restore_update_multi"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -145,6 +147,21 @@ class Zgr:
 
     def restore_update(self, seed: int, loss_plus: float, loss_minus: float, lr: float, stream=None) -> None:
         _check(lib().zgr_restore_update(self._h, seed, loss_plus, loss_minus, lr, _stream_ptr(stream)), "zgr_restore_update")
+
+    # -- several seeds in one sweep ---------------------------------------------------------------
+    def sweep_multi(self, seeds: Sequence[int], coeffs: Sequence[float], stream=None) -> None:
+        """theta <- rnd(theta + sum_i coeffs[i] z(seeds[i])) in one pass (zgr_sweep_multi)."""
+        n = len(seeds)
+        assert n == len(coeffs)
+        _check(lib().zgr_sweep_multi(self._h, n, (ctypes.c_uint64 * n)(*seeds), (ctypes.c_double * n)(*coeffs), _stream_ptr(stream)),
+               "zgr_sweep_multi")
+
+    def restore_update_multi(self, seeds: Sequence[int], loss_plus: Sequence[float], loss_minus: Sequence[float], lr: float, stream=None) -> None:
+        """Restore and projected-gradient update of several seeds in one pass (zgr_restore_update_multi)."""
+        n = len(seeds)
+        assert n == len(loss_plus) == len(loss_minus)
+        _check(lib().zgr_restore_update_multi(self._h, n, (ctypes.c_uint64 * n)(*seeds), (ctypes.c_double * n)(*loss_plus),
+                                              (ctypes.c_double * n)(*loss_minus), lr, _stream_ptr(stream)), "zgr_restore_update_multi")
 
     # -- compressed coefficients ----------------------------------------------------------------
     def set_coeffs_dtc(self, tensor: int, q, scale, zero=None, bits: int = 8) -> None:
@@ -215,6 +232,12 @@ class Zgr:
         act, seed, net = ctypes.c_int32(), ctypes.c_uint64(), ctypes.c_double()
         _check(lib().zgr_get_state(self._h, ctypes.byref(act), ctypes.byref(seed), ctypes.byref(net)), "zgr_get_state")
         return bool(act.value), seed.value, net.value
+
+    def active_seeds(self) -> int:
+        """Number of seeds whose perturbation is currently applied to the weights."""
+        act, seed, net = ctypes.c_int32(), ctypes.c_uint64(), ctypes.c_double()
+        _check(lib().zgr_get_state(self._h, ctypes.byref(act), ctypes.byref(seed), ctypes.byref(net)), "zgr_get_state")
+        return act.value
 
     def launch_count(self) -> int:
         return int(lib().zgr_launch_count(self._h))

@@ -124,6 +124,25 @@ class Pair:
                                        f"{what} tensor {l} {self.shapes[l]} r={self.ranks[l]}", operand=abs(c) * self.sigma_z(l)))
         return reports
 
+    def call_and_check_multi(self, seeds, coeffs, fn, what: str):
+        """Run one library call `fn()` that applies sum_q coeffs[q] z(seeds[q]); the oracle starts from the same theta."""
+        ots = [self.oracle_tensor(l) for l in range(len(self.shapes))]
+        before = [oracle.decode(t.theta, t.dtype) for t in ots]
+        fn()
+        torch.cuda.synchronize()
+        assert self.lib.device_status() == 0, "a kernel abandoned a bounded wait"
+        reports, exps = [], []
+        for l, t in enumerate(ots):
+            oracle.sweep_multi_tensor(t, seeds, coeffs, l, self.bits, self.a, self.b)
+            exps.append(oracle.decode(t.theta, t.dtype))
+        theta_max = max(max(np.abs(b).max(), np.abs(e).max()) for b, e in zip(before, exps))
+        operand = sum(abs(c) for c in coeffs)
+        for l, t in enumerate(ots):
+            got = to_double(self.theta[l])
+            reports.append(check_sweep(got, exps[l], before[l], self.dtype, theta_max,
+                                       f"{what} tensor {l} {self.shapes[l]} r={self.ranks[l]}", operand=operand * self.sigma_z(l)))
+        return reports
+
     def sigma_z(self, l: int) -> float:
         """rms size of z in tensor l: a^2 from the isotropic part, b^2 r/m from the guided part (U orthonormal)."""
         (m, n), r = self.shapes[l], self.ranks[l]
