@@ -83,6 +83,22 @@ def test_full_size_configuration_sampled_parity(name):
             if wl.dtype != "f32":
                 assert rep["equal"] > 0.9, (what, spec.name, rep)
         assert min(moved) > 0.3, (what, moved)       # no tensor was skipped by the sweep
+    # one pass with two seeds (zgr_sweep_multi), sampled the same way
+    seeds2, coeffs2 = [wl.seed(1, 0), wl.seed(1, 1)], [wl.eps, -0.5 * wl.eps]
+    before = {l: _gather(dm.theta[l], samples[l][1]) for l in picked}
+    z.sweep_multi(seeds2, coeffs2)
+    assert z.device_status() == 0
+    after = {l: _gather(dm.theta[l], samples[l][1]) for l in picked}
+    exps = {l: oracle.sweep_multi_elements(otens[l], before[l], seeds2, coeffs2, l, 16, a_o, b_o, samples[l][0]) for l in picked}
+    theta_max = max(max(np.abs(before[l]).max(), np.abs(exps[l]).max()) for l in picked)
+    for l in picked:
+        spec = wl.tensors[l]
+        sigma = float(np.sqrt(a_o**2 + b_o**2 * spec.rank / spec.rows))
+        rep = check_sweep(after[l], exps[l], before[l], wl.dtype, theta_max, f"{name} sweep_multi tensor {l} ({spec.name})",
+                          operand=1.5 * wl.eps * sigma)
+        assert rep["moved"] > 0.3, (spec.name, rep)
+    assert z.active_seeds() == 2
+    z.sweep_multi(seeds2, [-c for c in coeffs2])
     # nothing outside the model was touched and the state machine is idle again
     assert z.state()[0] is False
     z.close()
