@@ -125,9 +125,13 @@ int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, con
 
 /* Deliver the guided coefficients of one tensor compressed (Sec. 3.4, DTC): from now on
  *     G_l[k][c] = scale[k] * (q[k][c] - zero[k])       (x = lambda (x_quant - delta))
- * replaces the seed-drawn G_l.  q: device, rank x cols int8 row-major; scale: device, rank fp32;
- * zero: device, rank fp32, or NULL for delta = 0; bits must be 8.  Pointers are borrowed, not copied.
- * ZGR_EINVAL: bad tensor index, tensor without subspace, null q/scale, bits != 8.
+ * replaces the seed-drawn G_l.  scale: device, rank fp32; zero: device, rank fp32, or NULL for delta = 0.
+ *   bits = 8: q is device, rank x cols int8 (signed codes) row-major.
+ *   bits = 4: the paper's INT4 payload.  q is device, rank rows of (cols + 1)/2 bytes; each byte holds two
+ *             unsigned codes in [0, 15], the even column in the low nibble (the last byte of a row with an
+ *             odd number of columns has its high nibble ignored).  The zero point carries the offset.
+ * Pointers are borrowed, not copied.
+ * ZGR_EINVAL: bad tensor index, tensor without subspace, null q/scale, bits not 8 or 4.
  * ZGR_ESTATE: a perturbation is active (the coefficients must not change between a perturb and
  * its restore_update). */
 int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits);

@@ -251,6 +251,33 @@ def dtc_dequantise(q: np.ndarray, scale: np.ndarray, zero: Optional[np.ndarray] 
     return out
 
 
+def dtc_quantise_int4(G: np.ndarray):
+    """The paper's INT4 form of Sec. 3.4: unsigned codes x_q in [0, 15], lambda = (max - min)/15 and a zero
+    point delta per row, x = lambda (x_q - delta).  It is the affine quantiser above with codes and zero
+    point shifted by 8 from the signed range to the unsigned one (the dequantised values are the same)."""
+    q, sc, ze = dtc_quantise(G, bits=4, symmetric=False)
+    return (q.astype(np.int16) + 8).astype(np.int8), sc, (ze + np.float32(8.0)).astype(np.float32)
+
+
+def dtc_pack4(codes: np.ndarray) -> np.ndarray:
+    """Transmission layout of 4-bit codes: each row becomes (cols + 1)//2 bytes, column 2j in the low nibble
+    of byte j and column 2j + 1 in its high nibble (a missing last column is stored as 0)."""
+    codes = np.asarray(codes)
+    assert codes.ndim == 2 and codes.min() >= 0 and codes.max() <= 15
+    r, n = codes.shape
+    padded = np.zeros((r, 2 * ((n + 1) // 2)), dtype=np.uint8)
+    padded[:, :n] = codes
+    return (padded[:, 0::2] | (padded[:, 1::2] << 4)).astype(np.uint8)
+
+
+def dtc_unpack4(packed: np.ndarray, cols: int) -> np.ndarray:
+    packed = np.asarray(packed, dtype=np.uint8)
+    out = np.zeros((packed.shape[0], 2 * packed.shape[1]), dtype=np.int8)
+    out[:, 0::2] = packed & 15
+    out[:, 1::2] = packed >> 4
+    return out[:, :cols]
+
+
 # ----------------------------------------------------------------------------- the call sequence
 class OracleZGR:
     """Mirror of the library's call sequence over a list of :class:`OracleTensor`.

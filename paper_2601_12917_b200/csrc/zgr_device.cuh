@@ -252,9 +252,20 @@ __device__ __forceinline__ void coeffs8(const TensorDesc& td, const PhiloxKeys& 
   if (td.q != nullptr) {
     const float lambda = td.qscale[k] * cb;
     const float delta = td.qzero ? td.qzero[k] : 0.0f;
-    const int8_t* src = td.q + static_cast<int64_t>(k) * td.cols + c;
+    if (td.qbits == 4) {
+      // two unsigned 4-bit codes per byte, even column in the low nibble (c is a multiple of 8)
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(td.q) + static_cast<int64_t>(k) * ((td.cols + 1) >> 1) + (c >> 1);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) g[i] = lambda * (static_cast<float>(src[i]) - delta);
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t byte = src[i];
+        g[2 * i] = lambda * (static_cast<float>(byte & 15u) - delta);
+        g[2 * i + 1] = lambda * (static_cast<float>(byte >> 4) - delta);
+      }
+    } else {
+      const int8_t* src = td.q + static_cast<int64_t>(k) * td.cols + c;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) g[i] = lambda * (static_cast<float>(src[i]) - delta);
+    }
   } else {
     normals8<BITS, PRECISE>(keys, static_cast<uint32_t>(td.id), 1u, static_cast<uint64_t>(k) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(c),
                             unit, g);
@@ -267,7 +278,14 @@ template <int BITS, bool PRECISE>
 __device__ __forceinline__ float coeff1(const TensorDesc& td, const PhiloxKeys& keys, const NormalScale& unit, float cb, int k, int64_t c) {
   if (td.q != nullptr) {
     const float delta = td.qzero ? td.qzero[k] : 0.0f;
-    return td.qscale[k] * cb * (static_cast<float>(td.q[static_cast<int64_t>(k) * td.cols + c]) - delta);
+    float code;
+    if (td.qbits == 4) {
+      const uint32_t byte = reinterpret_cast<const uint8_t*>(td.q)[static_cast<int64_t>(k) * ((td.cols + 1) >> 1) + (c >> 1)];
+      code = static_cast<float>((c & 1) ? (byte >> 4) : (byte & 15u));
+    } else {
+      code = static_cast<float>(td.q[static_cast<int64_t>(k) * td.cols + c]);
+    }
+    return td.qscale[k] * cb * (code - delta);
   }
   return cb * normal1<BITS, PRECISE>(keys, static_cast<uint32_t>(td.id), 1u,
                                      static_cast<uint64_t>(k) * static_cast<uint64_t>(td.cols) + static_cast<uint64_t>(c), unit);

@@ -376,6 +376,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
     td.q = nullptr;
     td.qscale = nullptr;
     td.qzero = nullptr;
+    td.qbits = 8;
     td.rows = t.rows;
     td.cols = t.cols;
     td.rank = t.rank;
@@ -519,13 +520,14 @@ int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, con
 
 int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits) {
   if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
-  if (!q || !scale || bits != 8) return ZGR_EINVAL;
+  if (!q || !scale || (bits != 8 && bits != 4)) return ZGR_EINVAL;
   TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
   if (td.rank == 0) return ZGR_EINVAL;
   if (!ctx->ledger.empty()) return ZGR_ESTATE;
   td.q = q;
   td.qscale = scale;
   td.qzero = zero;
+  td.qbits = bits;
   ctx->descs_dirty = true;
   return ZGR_OK;
 }

@@ -12,7 +12,8 @@ struct TensorDesc {
   const float* U;        // rows x rank fp32 (caller's), or null
   const uint4* Ufrag;    // library-owned copy of U, split into bf16 hi/lo and laid out in the
                          // register order of the m16n8k16 A operand (tensor-core path only)
-  const int8_t* q;       // DTC codes rank x cols, or null -> coefficients drawn from the seed
+  const int8_t* q;       // DTC codes rank x cols (int8), or rank rows of (cols+1)/2 bytes holding two unsigned
+                         // 4-bit codes each, even column in the low nibble; null -> coefficients drawn from the seed
   const float* qscale;   // rank
   const float* qzero;    // rank or null
   int64_t rows, cols;
@@ -20,6 +21,7 @@ struct TensorDesc {
   int32_t kpad;          // r rounded up to the contraction width of the path in use
   int32_t id;            // generator tensor id (third counter word)
   int32_t dtype;
+  int32_t qbits;         // 8 or 4: width of the codes behind q
   int32_t umma;          // 1: served by the tcgen05 + TMA kernel (tensor maps and row-major hi/lo copies of U exist)
   void* Uhi;             // library-owned, rows_pad x kpad bf16 row-major (TMA source), or null
   void* Ulo;

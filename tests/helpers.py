@@ -92,11 +92,14 @@ class Pair:
         self.a, self.b = oracle.mix_scalars(alpha, self.d, self.K, scale_mode)
         self.theta_max = max(float(t.abs().max()) for t in self.theta)
 
-    def set_dtc(self, l: int, q: np.ndarray, scale: np.ndarray, zero=None):
+    def set_dtc(self, l: int, q: np.ndarray, scale: np.ndarray, zero=None, bits: int = 8):
+        """q: rank x cols codes (int8 for bits = 8, unsigned values 0..15 for bits = 4).  The oracle keeps the
+        codes as given; for bits = 4 the library receives them packed two to a byte (oracle.dtc_pack4)."""
         self.q[l] = torch.from_numpy(q).to(self.device)
         self.scale[l] = torch.from_numpy(scale).to(self.device)
         self.zero[l] = None if zero is None else torch.from_numpy(zero).to(self.device)
-        self.lib.set_coeffs_dtc(l, self.q[l], self.scale[l], self.zero[l])
+        payload = self.q[l] if bits == 8 else torch.from_numpy(oracle.dtc_pack4(q)).to(self.device)
+        self.lib.set_coeffs_dtc(l, payload, self.scale[l], self.zero[l], bits)
 
     def oracle_tensor(self, l: int) -> oracle.OracleTensor:
         (m, n) = self.shapes[l]

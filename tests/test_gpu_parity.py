@@ -189,6 +189,30 @@ def test_compressed_coefficients(dtype, rank, cols):
     p.step(seed=79, lp=2.0, lm=1.9, lr=1e-4)
 
 
+@pytest.mark.parametrize("dtype,rank,cols", [("f32", 8, 264), ("bf16", 32, 520), ("bf16", 64, 384), ("f16", 16, 1032), ("f16", 20, 101)])
+def test_int4_compressed_coefficients(dtype, rank, cols):
+    """The paper's INT4 payload (Sec. 3.4): unsigned 4-bit codes, two to a byte, with per-row scale and zero point."""
+    bits = 32 if dtype == "f32" else 16
+    p = Pair([(80, cols), (1, 30)], [rank, 0], dtype, seed=4, bits=bits)
+    G = oracle.coeffs(9, 0, bits, rank, cols)
+    q, sc, ze = oracle.dtc_quantise_int4(G)
+    p.set_dtc(0, q, sc, ze, bits=4)
+    reports = p.step(seed=77, lp=2.4, lm=1.6, lr=1e-4)
+    assert all(rep["moved"] > 0.3 for call in reports for rep in call)
+    # the guided part really comes from the codes: z moves by at most the quantisation bound from the seed-drawn one
+    if dtype == "f32":
+        z4 = to_double(p.lib.debug_z(9, 0)).reshape(80, cols)
+        p.q[0] = p.scale[0] = p.zero[0] = None
+        p.lib.clear_coeffs(0)
+        z_seed = to_double(p.lib.debug_z(9, 0)).reshape(80, cols)
+        U = p.U[0].cpu().numpy().astype(np.float64)
+        bound = p.b * (np.abs(U) @ np.tile(0.5 * sc[:, None].astype(np.float64), (1, cols)))
+        assert np.all(np.abs(z4 - z_seed) <= bound * 1.001 + 1e-4) and np.abs(z4 - z_seed).max() > 0
+    with pytest.raises(zgr.ZgrError) as e:
+        p.lib.set_coeffs_dtc(0, torch.zeros(rank, cols, dtype=torch.int8, device="cuda"), torch.ones(rank, device="cuda"), None, 5)
+    assert e.value.code == zgr.EINVAL
+
+
 def test_dtc_path_agrees_with_quantised_seed_coefficients():
     # quantise the seed-drawn G with the oracle's quantiser (Sec. 3.4) and feed it back compressed:
     # z must move by at most the quantisation bound

@@ -191,3 +191,28 @@ def test_dtc_coefficients_replace_seeded_ones():
     q2, sc2, ze2 = oracle.dtc_quantise(G2, 8, False)
     t2 = oracle.OracleTensor(np.zeros(m * n), m, n, oracle.F64, U=U, q=q2, scale=sc2, zero=ze2)
     np.testing.assert_allclose(oracle.z_tensor(t2, 3, 0, 32, a, b), U.astype(np.float64) @ oracle.dtc_dequantise(q2, sc2, ze2), atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- INT4 payload (Sec. 3.4)
+def test_int4_quantiser_error_bound_and_code_range():
+    rng = np.random.default_rng(5)
+    G = rng.standard_normal((6, 101))
+    q, sc, ze = oracle.dtc_quantise_int4(G)
+    assert q.min() >= 0 and q.max() <= 15                       # x_quant in [0, 2^b - 1]
+    for k in range(6):
+        lam = float(sc[k])
+        assert lam == pytest.approx((G[k].max() - G[k].min()) / 15.0, rel=1e-6)    # lambda = (max - min)/(2^b - 1)
+    back = oracle.dtc_dequantise(q, sc, ze)
+    assert np.all(np.abs(back - G) <= 0.5 * sc[:, None].astype(np.float64) * (1 + 1e-6) + 1e-12)   # |x - x'| <= lambda/2
+    assert {0, 15} <= set(np.unique(q))                         # both ends of the range are used
+
+
+def test_int4_packing_layout():
+    codes = np.array([[1, 2, 3, 4, 5], [15, 0, 9, 8, 7]], dtype=np.int8)
+    packed = oracle.dtc_pack4(codes)
+    # column 2j in the low nibble, column 2j+1 in the high nibble; the odd tail is padded with 0
+    assert packed.tolist() == [[0x21, 0x43, 0x05], [0x0F, 0x89, 0x07]]
+    assert np.array_equal(oracle.dtc_unpack4(packed, 5), codes)
+    rng = np.random.default_rng(6)
+    c = rng.integers(0, 16, size=(7, 64)).astype(np.int8)
+    assert np.array_equal(oracle.dtc_unpack4(oracle.dtc_pack4(c), 64), c)
