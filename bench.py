@@ -35,21 +35,26 @@ UNIT = "params/s"
 
 
 # DRAM traffic per launch of the dominant kernel from one ncu capture (profiles/sweep_umma_bf16_k32_llama7b.md:
-# small case, scaled by the elements processed), valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.77e9,
-               "source": "paper_2601_12917_b200/csrc/zgr_umma.cu", "sha1": "32fd37079633d0ec5c0ed9fdc10071367403bf7d"}
+# small case, scaled by the elements processed), valid only for the kernel sources it was taken from.
+NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.74e9,
+               "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
+                           "paper_2601_12917_b200/csrc/zgr_internal.h"],
+               "sha1": "d82c6e23644bb086301e24aff799031fb9a2b6e0"}
 
 
 def ncu_traffic(kernel: str, workload: str):
     import hashlib
     if kernel != NCU_TRAFFIC["kernel"] or workload != NCU_TRAFFIC["workload"]:
         return None
+    h = hashlib.sha1()
     try:
-        with open(os.path.join(ROOT, NCU_TRAFFIC["source"]), "rb") as f:
-            if hashlib.sha1(f.read()).hexdigest() != NCU_TRAFFIC["sha1"]:
-                return None           # the kernel has changed since the counters were taken
+        for src in NCU_TRAFFIC["sources"]:
+            with open(os.path.join(ROOT, src), "rb") as f:
+                h.update(f.read())
     except OSError:
         return None
+    if h.hexdigest() != NCU_TRAFFIC["sha1"]:
+        return None                   # the kernel has changed since the counters were taken
     return NCU_TRAFFIC["bytes_per_launch"]
 
 
