@@ -102,3 +102,51 @@ def test_full_size_configuration_sampled_parity(name):
     # nothing outside the model was touched and the state machine is idle again
     assert z.state()[0] is False
     z.close()
+
+
+@pytest.mark.parametrize("dtype,rows,cols,rank", [
+    ("bf16", 34000, 131072, 16),     # tcgen05 kernel, 4.46e9 elements: element indices beyond 2^32
+    ("f32", 1100, 4194304, 8),       # CUDA-core kernel, 4.61e9 elements, very long rows
+    ("bf16", 1, 4400000008, 0),      # isotropic kernel on one vector of 4.4e9 elements
+])
+def test_tensor_with_more_than_2_pow_32_elements(dtype, rows, cols, rank):
+    """Largest sizes: linear element indices, generator block indices and byte offsets all pass 2^32.
+    Sampled parity of one perturbation, with the samples concentrated at the far end of the tensor."""
+    tdt = {"bf16": torch.bfloat16, "f32": torch.float32}[dtype]
+    numel = rows * cols
+    need = numel * (2 if dtype == "bf16" else 4) * 1.1 + 2e9
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        pytest.skip(f"needs {need / 1e9:.0f} GB of free device memory")
+    assert numel > 2**32
+    g = torch.Generator(device="cuda").manual_seed(1)
+    w = torch.empty((rows, cols) if rows > 1 else (cols,), dtype=tdt, device="cuda")
+    chunk = 1 << 28
+    flat = w.view(-1)
+    for s in range(0, numel, chunk):                                  # N(0, 0.02^2) in slabs (bounded temporaries)
+        n = min(chunk, numel - s)
+        flat[s:s + n] = (0.02 * torch.randn(n, generator=g, device="cuda", dtype=torch.float32)).to(tdt)
+    U = None
+    if rank:
+        qmat, _ = torch.linalg.qr(torch.randn(rows, rank, generator=g, device="cuda", dtype=torch.float64))
+        U = qmat.to(torch.float32).contiguous()
+    eps = 1e-3
+    z = zgr.Zgr([w], [U], 0.5, eps, zgr.SCALE_UNIT, 16)
+    a_o, b_o = oracle.mix_scalars(0.5, numel, rank * cols, oracle.SCALE_UNIT)
+    rng = np.random.default_rng(0)
+    idx = np.unique(np.concatenate([rng.integers(0, numel, 4000), rng.integers(2**32, numel, 12000),
+                                    np.arange(numel - 2048, numel), np.arange(2**32 - 1024, 2**32 + 1024)])).astype(np.int64)
+    didx = torch.from_numpy(idx).cuda()
+    ot = oracle.OracleTensor(theta=np.zeros(0, dtype=np.float32), rows=rows, cols=cols, dtype=ORACLE_DTYPE[dtype],
+                             U=None if U is None else U.cpu().numpy())
+    before = _gather(w, didx)
+    z.perturb(99, eps)
+    assert z.device_status() == 0
+    after = _gather(w, didx)
+    exp = oracle.sweep_elements(ot, before, 99, 0, 16, a_o, b_o, eps, idx)
+    sigma = float(np.sqrt(a_o**2 + b_o**2 * rank / rows))
+    rep = check_sweep(after, exp, before, dtype, float(max(np.abs(before).max(), np.abs(exp).max())), f"{rows}x{cols} r={rank}",
+                      operand=eps * sigma)
+    assert rep["moved"] > 0.3, rep
+    z.restore_update(99, 2.0, 2.0, 0.0)
+    z.close()
