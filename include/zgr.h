@@ -123,6 +123,14 @@ int zgr_sweep_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, const double
 int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, const double* loss_plus, const double* loss_minus, double lr,
                              void* stream);
 
+/* Change the mixing ratio alpha of Eq. (perturbation) between steps; a and b are recomputed as in
+ * zgr_init.  This is the hook for the adaptive choice of the ZGR parameter mentioned in Sec. 1 ("based on
+ * the relative scales of BP-based and ZOO-based perturbations"): the paper gives no rule, so the caller
+ * applies its own to the norms of zgr_get_stats and sets the result here.
+ * ZGR_EINVAL: alpha outside [0, 1].  ZGR_ESTATE: a perturbation is active, or the context was built with
+ * alpha = 1 (its sweep plan carries no subspace operands) and alpha < 1 is asked for. */
+int zgr_set_alpha(zgr_ctx* ctx, double alpha);
+
 /* Deliver the guided coefficients of one tensor compressed (Sec. 3.4, DTC): from now on
  *     G_l[k][c] = scale[k] * (q[k][c] - zero[k])       (x = lambda (x_quant - delta))
  * replaces the seed-drawn G_l.  scale: device, rank fp32; zero: device, rank fp32, or NULL for delta = 0.
@@ -179,6 +187,21 @@ int zgr_tensor_norms_noalloc(zgr_ctx* ctx, uint64_t seed, int32_t tensor, double
 int zgr_debug_philox(zgr_ctx* ctx, uint64_t seed, int32_t tensor, int32_t tag, uint64_t first_block, int64_t n_blocks,
                      uint32_t* dev_out, void* stream);
 int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, void* stream);
+
+/* The work plan of a sweep, computed on the host alone (no device is needed or touched): which kernel
+ * family serves which part of which tensor.  Test hook for the planner: the items of a plan must cover
+ * every element of every tensor exactly once.  path: 0 isotropic (elements [row0_or_e0, +nrows_or_count) of
+ * the tensor), otherwise rows [row0_or_e0, +nrows_or_count) x columns [col0, +ncols): 1 CUDA-core rank <= 8,
+ * 2 legacy tensor-core, 3 fallback, 4 tcgen05.  `tensors[].data / U` are only inspected for alignment and
+ * null-ness.  tcgen05 != 0 plans as on a device where tensor maps can be made; multi != 0 gives the plan of
+ * the multi-seed sweeps.  Up to max_items items are written to out; *n_items receives the full count.
+ * Errors as zgr_init (ZGR_EINVAL), plus sm_count < 1 or a null n_items. */
+typedef struct {
+  int32_t path, kpad, tensor, ncols;
+  int64_t row0_or_e0, nrows_or_count, col0;
+} zgr_plan_item;
+int zgr_debug_plan(const zgr_tensor* tensors, int32_t n, const zgr_config* cfg, int32_t sm_count, int32_t tcgen05, int32_t multi,
+                   zgr_plan_item* out, int64_t max_items, int64_t* n_items);
 
 /* Per-kernel timing.  While enabled, every sweep launch is bracketed by CUDA events on its stream.
  * zgr_profile_read synchronises the device, writes one entry per kernel family that ran since the

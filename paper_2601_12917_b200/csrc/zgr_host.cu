@@ -50,6 +50,7 @@ struct zgr_ctx {
   double* d_stats = nullptr;
   std::map<uint64_t, double> ledger;  // seeds whose perturbation is applied to the weights -> sum of the coefficients applied
   uint64_t last_seed = 0;             // most recently swept seed (introspection)
+  bool guided_at_init = false;        // b != 0 when the sweep plan was made
   std::vector<Group> groups_multi;    // plan of multi-seed sweeps when it differs from `groups` (legacy tensor-core path only)
   bool multi_planned = false;
   int sticky = 0;                     // first CUDA failure, returned by every later call
@@ -278,6 +279,42 @@ int flush_descs(zgr_ctx* ctx, cudaStream_t st) {
 
 bool is_finite(double x) { return std::isfinite(x); }
 
+// Mixing scalars of Eq. (perturbation) with n := d and m := K
+void set_mixing(zgr_ctx* ctx, double alpha) {
+  const double d = static_cast<double>(ctx->d), K = static_cast<double>(ctx->K);
+  ctx->cfg.alpha = alpha;
+  ctx->a = std::sqrt(alpha / d);
+  ctx->b = ctx->K > 0 ? std::sqrt((1.0 - alpha) / K) : 0.0;
+  if (ctx->cfg.scale_mode == ZGR_SCALE_UNIT) {
+    ctx->a *= std::sqrt(d);
+    ctx->b *= std::sqrt(d);
+  }
+}
+
+// Argument checks shared by zgr_init and zgr_debug_plan; d = parameters, K = guided coefficients.
+int validate_model(const zgr_tensor* tensors, int32_t n, const zgr_config* cfg, int64_t* d_out, int64_t* K_out) {
+  if (!tensors || !cfg || n <= 0) return ZGR_EINVAL;
+  if (!(cfg->alpha >= 0.0 && cfg->alpha <= 1.0) || !is_finite(cfg->eps) || !(cfg->eps > 0.0)) return ZGR_EINVAL;
+  if (cfg->scale_mode != ZGR_SCALE_PAPER && cfg->scale_mode != ZGR_SCALE_UNIT) return ZGR_EINVAL;
+  if (cfg->bits_per_normal != 32 && cfg->bits_per_normal != 16) return ZGR_EINVAL;
+  int64_t d = 0, K = 0;
+  for (int32_t l = 0; l < n; ++l) {
+    const zgr_tensor& t = tensors[l];
+    if (!t.data || t.rows < 1 || t.cols < 1) return ZGR_EINVAL;
+    if (t.dtype != ZGR_F32 && t.dtype != ZGR_F16 && t.dtype != ZGR_BF16) return ZGR_EINVAL;
+    if (t.rank < 0 || t.rank > ZGR_MAX_RANK) return ZGR_EINVAL;
+    if ((t.rank == 0) != (t.U == nullptr)) return ZGR_EINVAL;
+    if (reinterpret_cast<uintptr_t>(t.data) % dtype_bytes(t.dtype) != 0) return ZGR_EINVAL;
+    if (t.U && reinterpret_cast<uintptr_t>(t.U) % 4 != 0) return ZGR_EINVAL;
+    if (t.rows > (INT64_MAX / t.cols)) return ZGR_EINVAL;
+    d += t.rows * t.cols;
+    K += static_cast<int64_t>(t.rank) * t.cols;
+  }
+  *d_out = d;
+  *K_out = K;
+  return ZGR_OK;
+}
+
 // Book-keeping of the coefficients applied under each seed; a seed whose coefficients cancel is idle again.
 void ledger_add(zgr_ctx* ctx, uint64_t seed, double c) {
   double& net = ctx->ledger[seed];
@@ -296,7 +333,7 @@ std::vector<Group>& multi_groups(zgr_ctx* ctx, int* rc) {
   if (!ctx->multi_planned) {
     std::vector<int> all(ctx->descs.size());
     for (size_t l = 0; l < all.size(); ++l) all[l] = static_cast<int>(l);
-    plan(ctx->descs, all, ctx->b != 0.0, ctx->cfg.bits_per_normal, ctx->sm_count, ctx->groups_multi, -1, true);
+    plan(ctx->descs, all, ctx->guided_at_init, ctx->cfg.bits_per_normal, ctx->sm_count, ctx->groups_multi, -1, true);
     *rc = upload_groups(ctx, ctx->groups_multi);
     ctx->multi_planned = true;
   }
@@ -325,36 +362,16 @@ extern "C" {
 int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_config* cfg) {
   if (!out) return ZGR_EINVAL;
   *out = nullptr;
-  if (!tensors || !cfg || n <= 0) return ZGR_EINVAL;
-  if (!(cfg->alpha >= 0.0 && cfg->alpha <= 1.0) || !is_finite(cfg->eps) || !(cfg->eps > 0.0)) return ZGR_EINVAL;
-  if (cfg->scale_mode != ZGR_SCALE_PAPER && cfg->scale_mode != ZGR_SCALE_UNIT) return ZGR_EINVAL;
-  if (cfg->bits_per_normal != 32 && cfg->bits_per_normal != 16) return ZGR_EINVAL;
   int64_t d = 0, K = 0;
-  for (int32_t l = 0; l < n; ++l) {
-    const zgr_tensor& t = tensors[l];
-    if (!t.data || t.rows < 1 || t.cols < 1) return ZGR_EINVAL;
-    if (t.dtype != ZGR_F32 && t.dtype != ZGR_F16 && t.dtype != ZGR_BF16) return ZGR_EINVAL;
-    if (t.rank < 0 || t.rank > ZGR_MAX_RANK) return ZGR_EINVAL;
-    if ((t.rank == 0) != (t.U == nullptr)) return ZGR_EINVAL;
-    if (reinterpret_cast<uintptr_t>(t.data) % dtype_bytes(t.dtype) != 0) return ZGR_EINVAL;
-    if (t.U && reinterpret_cast<uintptr_t>(t.U) % 4 != 0) return ZGR_EINVAL;
-    if (t.rows > (INT64_MAX / t.cols)) return ZGR_EINVAL;
-    d += t.rows * t.cols;
-    K += static_cast<int64_t>(t.rank) * t.cols;
-  }
+  const int valid = validate_model(tensors, n, cfg, &d, &K);
+  if (valid != ZGR_OK) return valid;
 
   zgr_ctx* ctx = new (std::nothrow) zgr_ctx();
   if (!ctx) return ZGR_ENOMEM;
   ctx->cfg = *cfg;
   ctx->d = d;
   ctx->K = K;
-  // Eq. (perturbation) with n := d and m := K
-  ctx->a = std::sqrt(cfg->alpha / static_cast<double>(d));
-  ctx->b = K > 0 ? std::sqrt((1.0 - cfg->alpha) / static_cast<double>(K)) : 0.0;
-  if (cfg->scale_mode == ZGR_SCALE_UNIT) {
-    ctx->a *= std::sqrt(static_cast<double>(d));
-    ctx->b *= std::sqrt(static_cast<double>(d));
-  }
+  set_mixing(ctx, cfg->alpha);
 
   int rc = check(ctx, cudaGetDevice(&ctx->device));
   if (rc == ZGR_OK) rc = check(ctx, cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device));
@@ -367,6 +384,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
   ctx->tmaps.resize(static_cast<size_t>(3 * n));
   std::memset(ctx->tmaps.data(), 0, ctx->tmaps.size() * sizeof(CUtensorMap));
   const bool guided_on = ctx->b != 0.0;
+  ctx->guided_at_init = guided_on;
   for (int32_t l = 0; l < n && rc == ZGR_OK; ++l) {
     const zgr_tensor& t = tensors[l];
     TensorDesc& td = ctx->descs[static_cast<size_t>(l)];
@@ -518,6 +536,17 @@ int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, con
   return ZGR_OK;
 }
 
+int zgr_set_alpha(zgr_ctx* ctx, double alpha) {
+  if (!ctx || !(alpha >= 0.0 && alpha <= 1.0)) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (!ctx->ledger.empty()) return ZGR_ESTATE;
+  // The kernels serving each tensor were chosen at zgr_init; a context built with alpha = 1 (no guided
+  // part at all) has no tensor-core operands and keeps serving every tensor without its subspace.
+  if (ctx->guided_at_init == false && alpha < 1.0 && ctx->K > 0) return ZGR_ESTATE;
+  set_mixing(ctx, alpha);
+  return ZGR_OK;
+}
+
 int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits) {
   if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
   if (!q || !scale || (bits != 8 && bits != 4)) return ZGR_EINVAL;
@@ -557,7 +586,7 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
     int64_t target = std::min<int64_t>(std::max<int64_t>(total / (static_cast<int64_t>(ctx->sm_count) * 64), 4096), 131072);
     for (size_t l = 0; l < n; ++l) {
       const TensorDesc& t = ctx->descs[l];
-      if (t.umma && ctx->b != 0.0) continue;
+      if (t.umma && ctx->guided_at_init) continue;
       for (int64_t c0 = 0; c0 < t.cols; c0 += 64) {
         const int ncols = static_cast<int>(std::min<int64_t>(64, t.cols - c0));
         const int64_t nrows = std::max<int64_t>(1, target / ncols);
@@ -626,7 +655,7 @@ int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, voi
   std::vector<TensorDesc> one(1, ctx->descs[static_cast<size_t>(tensor)]);
   one[0].data = dev_out;
   std::vector<Group> groups;
-  const bool guided_on = ctx->b != 0.0;
+  const bool guided_on = ctx->guided_at_init;
   plan(one, std::vector<int>(1, 0), guided_on, ctx->cfg.bits_per_normal, ctx->sm_count, groups, ZGR_F32);
   const size_t owned_before = ctx->owned.size();
   TensorDesc* d_one = nullptr;
@@ -665,6 +694,42 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
     if (rc == ZGR_OK) ctx->launches++;
   }
   return rc;
+}
+
+int zgr_debug_plan(const zgr_tensor* tensors, int32_t n, const zgr_config* cfg, int32_t sm_count, int32_t tcgen05, int32_t multi,
+                   zgr_plan_item* out, int64_t max_items, int64_t* n_items) {
+  if (!n_items || sm_count < 1 || max_items < 0 || (max_items > 0 && !out)) return ZGR_EINVAL;
+  int64_t d = 0, K = 0;
+  const int valid = validate_model(tensors, n, cfg, &d, &K);
+  if (valid != ZGR_OK) return valid;
+  const bool guided_on = K > 0 && cfg->alpha < 1.0;
+  std::vector<TensorDesc> descs(static_cast<size_t>(n));
+  std::vector<int> all(static_cast<size_t>(n));
+  for (int32_t l = 0; l < n; ++l) {
+    const zgr_tensor& t = tensors[l];
+    TensorDesc& td = descs[static_cast<size_t>(l)];
+    std::memset(&td, 0, sizeof(td));
+    td.data = t.data; td.U = t.U; td.rows = t.rows; td.cols = t.cols; td.rank = t.rank; td.id = l; td.dtype = t.dtype; td.qbits = 8;
+    const bool vec = (reinterpret_cast<uintptr_t>(t.data) & 15) == 0 && (t.cols % 8 == 0);
+    if (guided_on && t.rank > 8 && vec && t.dtype != ZGR_F32) {
+      // what zgr_init would have built for this tensor: operand copies for the tensor-core kernels
+      td.kpad = t.rank <= 16 ? 16 : (t.rank <= 32 ? 32 : 64);
+      td.Ufrag = reinterpret_cast<const uint4*>(uintptr_t{16});   // marker only: never dereferenced by the planner
+      td.umma = (tcgen05 && t.rows < (int64_t{1} << 31) - 256 && t.cols < (int64_t{1} << 31) - 256) ? 1 : 0;
+    }
+    all[static_cast<size_t>(l)] = l;
+  }
+  std::vector<Group> groups;
+  plan(descs, all, guided_on, cfg->bits_per_normal, sm_count, groups, -1, multi != 0);
+  int64_t count = 0;
+  for (const Group& g : groups)
+    for (const WorkItem& w : g.items) {
+      if (count < max_items)
+        out[count] = zgr_plan_item{g.kc.path, g.kc.kpad, w.tensor, w.ncols, w.row0_or_e0, w.nrows_or_count, w.col0};
+      ++count;
+    }
+  *n_items = count;
+  return ZGR_OK;
 }
 
 int zgr_profile(zgr_ctx* ctx, int32_t enable) {

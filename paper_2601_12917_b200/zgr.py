@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
         L.zgr_sweep_multi.argtypes = [vp, i32, ctypes.POINTER(u64), ctypes.POINTER(dbl), vp]
         L.zgr_restore_update_multi.argtypes = [vp, i32, ctypes.POINTER(u64), ctypes.POINTER(dbl), ctypes.POINTER(dbl), dbl, vp]
         L.zgr_set_coeffs_dtc.argtypes = [vp, i32, vp, vp, vp, i32]
+        L.zgr_set_alpha.argtypes = [vp, dbl]
         L.zgr_clear_coeffs.argtypes = [vp, i32]
         L.zgr_get_stats.argtypes = [vp, u64, ctypes.POINTER(dbl), vp]
         L.zgr_debug_philox.argtypes = [vp, u64, i32, i32, u64, i64, vp, vp]
@@ -84,7 +85,7 @@ def lib() -> ctypes.CDLL:
         L.zgr_strerror.restype = ctypes.c_char_p
         for name in ("zgr_init", "zgr_perturb", "zgr_restore_update", "zgr_set_coeffs_dtc", "zgr_clear_coeffs", "zgr_get_stats",
                      "zgr_debug_philox", "zgr_debug_z", "zgr_get_scalars", "zgr_get_state", "zgr_update_subspace", "zgr_profile",
-                     "zgr_profile_read", "zgr_sweep_multi", "zgr_restore_update_multi"):
+                     "zgr_profile_read", "zgr_sweep_multi", "zgr_restore_update_multi", "zgr_set_alpha"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -162,6 +163,10 @@ class Zgr:
         assert n == len(loss_plus) == len(loss_minus)
         _check(lib().zgr_restore_update_multi(self._h, n, (ctypes.c_uint64 * n)(*seeds), (ctypes.c_double * n)(*loss_plus),
                                               (ctypes.c_double * n)(*loss_minus), lr, _stream_ptr(stream)), "zgr_restore_update_multi")
+
+    def set_alpha(self, alpha: float) -> None:
+        """New mixing ratio for the following steps (zgr_set_alpha)."""
+        _check(lib().zgr_set_alpha(self._h, alpha), "zgr_set_alpha")
 
     # -- compressed coefficients ----------------------------------------------------------------
     def set_coeffs_dtc(self, tensor: int, q, scale, zero=None, bits: int = 8) -> None:

@@ -90,3 +90,34 @@ print(sorted(k["path"] for k in p.lib.profile_read()))
     r = subprocess.run([sys.executable, "-c", code, ROOT], env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stderr[-2000:]
     assert "'mma'" in r.stdout and "umma" not in r.stdout
+
+
+def test_set_alpha_between_steps():
+    """zgr_set_alpha recomputes the mixing scalars of Eq. (perturbation); the following sweeps and norms use them."""
+    p = Pair([(140, 520), (1, 64), (96, 256)], [32, 0, 8], "bf16", bits=16, seed=3, alpha=0.5)
+    p.step(seed=1, lp=2.0, lm=1.9, lr=1e-4)
+    for alpha in (0.2, 1.0, 0.0, 0.7):
+        p.lib.set_alpha(alpha)
+        p.alpha = alpha
+        p.a, p.b = oracle.mix_scalars(alpha, p.d, p.K, p.scale_mode)
+        a, b = p.lib.scalars()
+        assert a == pytest.approx(p.a, rel=1e-14) and b == pytest.approx(p.b, rel=1e-14)
+        p.step(seed=10 + int(alpha * 10), lp=2.2, lm=1.7, lr=1e-4)
+        got = p.lib.get_stats(5)
+        for l in range(3):
+            exp = oracle.stats_tensor(p.oracle_tensor(l), 5, l, p.bits, p.a, p.b)
+            np.testing.assert_allclose(got[l], exp, rtol=2e-5, atol=1e-12)
+    with pytest.raises(zgr.ZgrError) as e:
+        p.lib.set_alpha(1.5)
+    assert e.value.code == zgr.EINVAL
+    p.lib.perturb(3, 1e-3)
+    with pytest.raises(zgr.ZgrError) as e:
+        p.lib.set_alpha(0.5)
+    assert e.value.code == zgr.ESTATE
+    p.lib.restore_update(3, 2.0, 2.0, 0.0)
+    # a context built without a guided part cannot grow one
+    q = Pair([(64, 256)], [8], "f32", alpha=1.0)
+    with pytest.raises(zgr.ZgrError) as e:
+        q.lib.set_alpha(0.5)
+    assert e.value.code == zgr.ESTATE
+    q.lib.set_alpha(1.0)
