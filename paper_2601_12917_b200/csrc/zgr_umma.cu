@@ -477,7 +477,10 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       const uint64_t tcols = static_cast<uint64_t>(td.cols);   // kept in a register: the barriers below force reloads of anything read through td
       // ---- coefficient strips c b G -> K-major hi/lo operands, one per tile of a row block ----
       for (int idx = et; idx < (KP / 2) * (NSUB * NS / 8); idx += kEpiWarps * 32) {
-        const int kp = idx / (NSUB * NS / 8), o = idx % (NSUB * NS / 8);
+        // consecutive lanes take consecutive pairs of rows k of the same columns: their 32-bit stores below then
+        // fall into KP/2 consecutive words of one operand row (with the octet index fastest they would all hit
+        // one bank: 27 wavefronts per store instead of 2)
+        const int kp = idx % (KP / 2), o = idx / (KP / 2);
         const int cc = 8 * o;                       // column within the item's strip
         if (cc >= ((w.ncols + NS - 1) / NS) * NS) continue;   // tiles of this item that do not exist
         float g0[8], g1[8];
