@@ -215,7 +215,7 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 #define ZGR_S16 4
 #endif
 #ifndef ZGR_S32
-#define ZGR_S32 4
+#define ZGR_S32 5
 #endif
 #ifndef ZGR_S64
 #define ZGR_S64 4
@@ -224,7 +224,7 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 #define ZGR_N16 4
 #endif
 #ifndef ZGR_N32
-#define ZGR_N32 3
+#define ZGR_N32 2
 #endif
 #ifndef ZGR_N64
 #define ZGR_N64 1
