@@ -212,7 +212,7 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 #define ZGR_TILE_N32 128
 #endif
 #ifndef ZGR_S16
-#define ZGR_S16 4
+#define ZGR_S16 5
 #endif
 #ifndef ZGR_S32
 #define ZGR_S32 5
@@ -221,7 +221,7 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 #define ZGR_S64 4
 #endif
 #ifndef ZGR_N16
-#define ZGR_N16 4
+#define ZGR_N16 2
 #endif
 #ifndef ZGR_N32
 #define ZGR_N32 2
