@@ -51,6 +51,7 @@ struct zgr_ctx {
   std::map<uint64_t, double> ledger;  // seeds whose perturbation is applied to the weights -> sum of the coefficients applied
   uint64_t last_seed = 0;             // most recently swept seed (introspection)
   bool guided_at_init = false;        // b != 0 when the sweep plan was made
+  std::vector<char> frag_stale;       // per tensor: the fragment-order copy of U (legacy tensor-core kernel) lags behind U
   std::vector<Group> groups_multi;    // plan of multi-seed sweeps when it differs from `groups` (legacy tensor-core path only)
   bool multi_planned = false;
   int sticky = 0;                     // first CUDA failure, returned by every later call
@@ -381,6 +382,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
   }
 
   ctx->descs.resize(static_cast<size_t>(n));
+  ctx->frag_stale.assign(static_cast<size_t>(n), 0);
   ctx->tmaps.resize(static_cast<size_t>(3 * n));
   std::memset(ctx->tmaps.data(), 0, ctx->tmaps.size() * sizeof(CUtensorMap));
   const bool guided_on = ctx->b != 0.0;
@@ -651,6 +653,13 @@ int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, voi
   if (reinterpret_cast<uintptr_t>(dev_out) % 4 != 0) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (ctx->frag_stale[static_cast<size_t>(tensor)]) {
+    const TensorDesc& cur = ctx->descs[static_cast<size_t>(tensor)];
+    const int rcf = check(ctx, launch_split_subspace(cur.U, cur.rows, cur.rank, cur.kpad, const_cast<uint4*>(cur.Ufrag), st));
+    if (rcf != ZGR_OK) return rcf;
+    ctx->launches++;
+    ctx->frag_stale[static_cast<size_t>(tensor)] = 0;
+  }
   // a one-tensor model whose weights are the zeroed output buffer, swept once with scale 1
   std::vector<TensorDesc> one(1, ctx->descs[static_cast<size_t>(tensor)]);
   one[0].data = dev_out;
@@ -685,8 +694,14 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
     if (rc != ZGR_OK) return rc;
   }
   if (td.Ufrag != nullptr) {
-    rc = check(ctx, launch_split_subspace(td.U, td.rows, td.rank, td.kpad, const_cast<uint4*>(td.Ufrag), st));
-    if (rc == ZGR_OK) ctx->launches++;
+    if (td.umma) {
+      // the sweeps of this tensor read the row-major copy below; the fragment-order copy is only needed by
+      // zgr_debug_z and is rebuilt there on demand
+      ctx->frag_stale[static_cast<size_t>(tensor)] = 1;
+    } else {
+      rc = check(ctx, launch_split_subspace(td.U, td.rows, td.rank, td.kpad, const_cast<uint4*>(td.Ufrag), st));
+      if (rc == ZGR_OK) ctx->launches++;
+    }
   }
   if (rc == ZGR_OK && td.umma) {
     const int64_t rows_pad = ((td.rows + 127) / 128) * 128;
