@@ -229,6 +229,12 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 #ifndef ZGR_N64
 #define ZGR_N64 1
 #endif
+// Epilogue groups: 1 = every epilogue warp works on every tile (32 rows x 32 columns each); 2 = two groups of
+// warps take alternate tiles (32 rows x 64 columns each, in two passes), so that one group's per-tile waits
+// fall under the other group's arithmetic.
+#ifndef ZGR_GROUPS
+#define ZGR_GROUPS 2
+#endif
 template <int KP>
 struct UmmaCfg {
   static constexpr int NS = KP == 64 ? 128 : (KP == 32 ? ZGR_TILE_N32 : ZGR_TILE_N16);   // columns per tile / per accumulator buffer
@@ -296,13 +302,14 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
+    constexpr int kWarpsPerTile = kEpiWarps / ((ZGR_GROUPS == 2 && NS == 128) ? 2 : 1);   // epilogue warps that work on one tile
     for (int s = 0; s < S; ++s) {
       mbar_init(BAR_FULL(s), 1);
-      mbar_init(BAR_OUT(s), kEpiWarps);
+      mbar_init(BAR_OUT(s), kWarpsPerTile);
     }
     for (int b = 0; b < NACC; ++b) {
       mbar_init(BAR_ACC_FULL(b), 1);
-      mbar_init(BAR_ACC_EMPTY(b), kEpiWarps);
+      mbar_init(BAR_ACC_EMPTY(b), kWarpsPerTile);
     }
     for (int u = 0; u < US; ++u) {
       mbar_init(BAR_U_FULL(u), 1);
@@ -458,13 +465,13 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
     // Warp (quad, cgrp) owns rows 32 quad .. 32 quad + 31 and columns 32 cgrp .. 32 cgrp + 31 of every tile.
     const int e = warp - 2;                 // 0..15
     const int quad = warp & 3;              // tensor-memory lane quadrant this warp may read
-    const int cgrp = e >> 2;                // which 32 columns of the tile
+    constexpr int GROUPS = (ZGR_GROUPS == 2 && NS == 128) ? 2 : 1;
+    const int grp = GROUPS == 2 ? (e >> 3) : 0;                              // which tiles: t % GROUPS == grp
+    const int cg_first = GROUPS == 2 ? 2 * ((e >> 2) & 1) : (e >> 2);        // first 32-column group of this warp
     const int et = e * 32 + lane;
-    const uint32_t tmem_warp = tmem_base + (static_cast<uint32_t>(32 * quad) << 16) + static_cast<uint32_t>(32 * cgrp);
+    const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(32 * quad) << 16);
     const int row_in_tile = 32 * quad + lane;
     const uint32_t row_xor = static_cast<uint32_t>(row_in_tile & 7);
-    const uint32_t chunk0 = static_cast<uint32_t>(((32 * cgrp) & 63) >> 3);
-    const uint32_t out_off = static_cast<uint32_t>(((32 * cgrp) >> 6) * 16384 + row_in_tile * 128);
     const uint32_t theta_s32 = smem_u32(theta_base);
     const uint32_t g_s32 = smem_u32(g_base);
     int t = 0, item_no = 0;
@@ -475,6 +482,13 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       const uint32_t tid = static_cast<uint32_t>(td.id);
       const int r = td.rank;
       const uint64_t tcols = static_cast<uint64_t>(td.cols);   // kept in a register: the barriers below force reloads of anything read through td
+      if (GROUPS == 2 && t > 0) {
+        // The strips are about to be overwritten.  With two groups this warp may be one tile ahead of the
+        // other group, whose last tile of the previous item can still have products in flight that read the
+        // old strips: wait until that tile's accumulator is complete (no later product exists before BAR_G).
+        const int tp = t - 1;
+        if (!mbar_wait<false>(BAR_ACC_FULL(tp % NACC), (tp / NACC) & 1, abort_flag, error, 11)) break;
+      }
       // ---- coefficient strips c b G -> K-major hi/lo operands, one per tile of a row block ----
       for (int idx = et; idx < (KP / 2) * (NSUB * NS / 8); idx += kEpiWarps * 32) {
         // consecutive lanes take consecutive pairs of rows k of the same columns: their 32-bit stores below then
@@ -514,18 +528,26 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       // point: first the integer rounds of the generator, then the special-function half of the
       // transform.  Holding every other column group back once per item puts half of each scheduler's
       // warps in the other phase, so the two pipes overlap (measured: 6.5 -> 6.15 ms per 7B sweep).
-      if (cgrp & 1) __nanosleep(kStaggerNs);
+      if (GROUPS == 1 && (cg_first & 1)) __nanosleep(kStaggerNs);
 
       const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
       const int nsub = (w.ncols + NS - 1) / NS;
       double sum_iso = 0.0, sum_gd = 0.0, sum_z = 0.0;   // STATS only
       for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128) {
         const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
-        const uint64_t row_e = static_cast<uint64_t>(row) * tcols + static_cast<uint64_t>(w.col0 + 32 * cgrp);
+        const uint64_t row_e0 = static_cast<uint64_t>(row) * tcols + static_cast<uint64_t>(w.col0);
         for (int sub = 0; sub < nsub; ++sub, ++t) {
+          if (GROUPS == 2 && (t & 1) != grp) continue;     // the other group's tile
           const int s = t % S, b = t % NACC;
           if (!mbar_wait<false>(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
           tc_fence_after();
+#pragma unroll
+          for (int pass = 0; pass < GROUPS; ++pass) {
+          const int cgrp = cg_first + pass;                // which 32 columns of the tile
+          const uint32_t tmem_warp = tmem_row + static_cast<uint32_t>(32 * cgrp);
+          const uint32_t chunk0 = static_cast<uint32_t>(((32 * cgrp) & 63) >> 3);
+          const uint32_t out_off = static_cast<uint32_t>(((32 * cgrp) >> 6) * 16384 + row_in_tile * 128);
+          const uint64_t row_e = row_e0 + static_cast<uint64_t>(32 * cgrp);
           if (NS * sub + 32 * cgrp < w.ncols) {
             const uint64_t oct0 = (row_e + static_cast<uint64_t>(NS * sub)) >> 3;
             const uint32_t oct0_lo = static_cast<uint32_t>(oct0), oct0_hi = static_cast<uint32_t>(oct0 >> 32);
@@ -576,6 +598,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
               sts128(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4), q);
             }
             }
+          }
           }
           tc_fence_before();
           fence_proxy_async();

@@ -304,3 +304,16 @@ def test_norm_bookkeeping(bits):
         np.testing.assert_allclose(got[l], exp, rtol=2e-5, atol=1e-12)
     # the weights were not touched
     assert p.lib.state()[0] is False
+
+
+@pytest.mark.parametrize("dtype,rows,cols,rank", [("f16", 16384, 2048, 16), ("bf16", 8192, 4096, 32), ("bf16", 6144, 1536, 64)])
+def test_many_work_items_per_block(dtype, rows, cols, rank):
+    """Tensors cut into ~1000 small work items, several per persistent block: the hand-over between items
+    (coefficient strips rewritten while the pipeline still holds tiles of the previous item) is exercised
+    hundreds of times per launch.  Every element is compared with the oracle."""
+    p = Pair([(rows, cols)], [rank], dtype, bits=16, seed=21)
+    reports = p.step(seed=12, lp=2.3, lm=1.8, lr=1e-4)
+    for call in reports:
+        assert call[0]["moved"] > 0.3 and call[0]["equal"] > 0.9, call
+    seeds, coeffs = [31, 32], [1e-3, -7e-4]
+    p.call_and_check_multi(seeds, coeffs, lambda: p.lib.sweep_multi(seeds, coeffs), "sweep_multi")
