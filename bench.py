@@ -36,10 +36,10 @@ UNIT = "params/s"
 
 # DRAM traffic per launch of the dominant kernel from one ncu capture (profiles/sweep_umma_bf16_k32_llama7b.md:
 # small case, scaled by the elements processed), valid only for the kernel sources it was taken from.
-NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.77e9,
+NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.76e9,
                "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
                            "paper_2601_12917_b200/csrc/zgr_internal.h"],
-               "sha1": "8789bef4c519b2bb699ed585654a736ee80da088"}
+               "sha1": "321529081483383425cfc4fd6095c9b34cf07f07"}
 
 
 def ncu_traffic(kernel: str, workload: str):

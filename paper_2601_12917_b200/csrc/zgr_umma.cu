@@ -212,7 +212,7 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 #define ZGR_TILE_N32 128
 #endif
 #ifndef ZGR_S16
-#define ZGR_S16 5
+#define ZGR_S16 6
 #endif
 #ifndef ZGR_S32
 #define ZGR_S32 5
