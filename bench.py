@@ -39,7 +39,7 @@ UNIT = "params/s"
 NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.76e9,
                "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
                            "paper_2601_12917_b200/csrc/zgr_internal.h"],
-               "sha1": "321529081483383425cfc4fd6095c9b34cf07f07"}
+               "sha1": "3b6fd45df0ef010a65380e67ed1c8d37b3f9ba01"}
 
 
 def ncu_traffic(kernel: str, workload: str):

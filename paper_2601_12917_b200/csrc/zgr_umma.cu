@@ -229,9 +229,9 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 #ifndef ZGR_N64
 #define ZGR_N64 1
 #endif
-// Epilogue groups: 1 = every epilogue warp works on every tile (32 rows x 32 columns each); 2 = two groups of
-// warps take alternate tiles (32 rows x 64 columns each, in two passes), so that one group's per-tile waits
-// fall under the other group's arithmetic.
+// Epilogue groups: 1 = every epilogue warp works on every tile (32 rows x 32 columns each); 2 (4) = two (four)
+// groups of warps take tiles in turn (32 rows x 64 (128) columns each, in two (four) passes), so that one group's
+// per-tile waits fall under the other groups' arithmetic.
 #ifndef ZGR_GROUPS
 #define ZGR_GROUPS 2
 #endif
@@ -241,6 +241,7 @@ struct UmmaCfg {
   static constexpr bool WIDE = NS > 128;
   static constexpr int EPI_WARPS = NS / 8;                 // one epilogue warp per 32 rows x 32 columns of a tile
   static constexpr int THREADS = 32 * (2 + EPI_WARPS);
+  static constexpr int GROUPS = NS == 128 ? ZGR_GROUPS : 1;   // epilogue groups on alternate tiles (1, 2 or 4; see ZGR_GROUPS)
   static constexpr int NSUB = KP == 64 ? ZGR_N64 : (KP == 32 ? ZGR_N32 : ZGR_N16);   // adjacent tiles per row block that share one U tile
   static constexpr int STAGES = KP == 64 ? ZGR_S64 : (KP == 32 ? ZGR_S32 : ZGR_S16);  // theta tiles in flight (loaded, transformed in place, stored)
   static constexpr int USTAGES = 2;                        // U tiles in flight
@@ -302,7 +303,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    constexpr int kWarpsPerTile = kEpiWarps / ((ZGR_GROUPS == 2 && NS == 128) ? 2 : 1);   // epilogue warps that work on one tile
+    constexpr int kWarpsPerTile = kEpiWarps / Cfg::GROUPS;   // epilogue warps that work on one tile
     for (int s = 0; s < S; ++s) {
       mbar_init(BAR_FULL(s), 1);
       mbar_init(BAR_OUT(s), kWarpsPerTile);
@@ -465,9 +466,9 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
     // Warp (quad, cgrp) owns rows 32 quad .. 32 quad + 31 and columns 32 cgrp .. 32 cgrp + 31 of every tile.
     const int e = warp - 2;                 // 0..15
     const int quad = warp & 3;              // tensor-memory lane quadrant this warp may read
-    constexpr int GROUPS = (ZGR_GROUPS == 2 && NS == 128) ? 2 : 1;
-    const int grp = GROUPS == 2 ? (e >> 3) : 0;                              // which tiles: t % GROUPS == grp
-    const int cg_first = GROUPS == 2 ? 2 * ((e >> 2) & 1) : (e >> 2);        // first 32-column group of this warp
+    constexpr int GROUPS = Cfg::GROUPS;                                      // each warp covers GROUPS column groups of its tiles
+    const int grp = e / (kEpiWarps / GROUPS);                                // which tiles: t % GROUPS == grp
+    const int cg_first = ((e >> 2) % (kEpiWarps / 4 / GROUPS)) * GROUPS;     // first 32-column group of this warp
     const int et = e * 32 + lane;
     const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(32 * quad) << 16);
     const int row_in_tile = 32 * quad + lane;
@@ -482,7 +483,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       const uint32_t tid = static_cast<uint32_t>(td.id);
       const int r = td.rank;
       const uint64_t tcols = static_cast<uint64_t>(td.cols);   // kept in a register: the barriers below force reloads of anything read through td
-      if (GROUPS == 2 && t > 0) {
+      if (GROUPS > 1 && t > 0) {
         // The strips are about to be overwritten.  With two groups this warp may be one tile ahead of the
         // other group, whose last tile of the previous item can still have products in flight that read the
         // old strips: wait until that tile's accumulator is complete (no later product exists before BAR_G).
@@ -537,7 +538,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
         const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
         const uint64_t row_e0 = static_cast<uint64_t>(row) * tcols + static_cast<uint64_t>(w.col0);
         for (int sub = 0; sub < nsub; ++sub, ++t) {
-          if (GROUPS == 2 && (t & 1) != grp) continue;     // the other group's tile
+          if (GROUPS > 1 && (t % GROUPS) != grp) continue;     // another group's tile
           const int s = t % S, b = t % NACC;
           if (!mbar_wait<false>(BAR_ACC_FULL(b), (t / NACC) & 1, abort_flag, error, 6)) { ok = false; break; }
           tc_fence_after();
