@@ -39,7 +39,15 @@ UNIT = "params/s"
 NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.76e9,
                "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
                            "paper_2601_12917_b200/csrc/zgr_internal.h"],
-               "sha1": "3b6fd45df0ef010a65380e67ed1c8d37b3f9ba01"}
+               "sha1": "34e2c55264b480439074b4fc8f445f816e3226fe"}
+
+
+def _code_only(text: str) -> str:
+    """Source text without comments and white space: the digest below follows the code, not its commentary."""
+    import re
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"//[^\n]*", "", text)
+    return re.sub(r"\s+", "", text)
 
 
 def ncu_traffic(kernel: str, workload: str):
@@ -49,8 +57,8 @@ def ncu_traffic(kernel: str, workload: str):
     h = hashlib.sha1()
     try:
         for src in NCU_TRAFFIC["sources"]:
-            with open(os.path.join(ROOT, src), "rb") as f:
-                h.update(f.read())
+            with open(os.path.join(ROOT, src), "r") as f:
+                h.update(_code_only(f.read()).encode())
     except OSError:
         return None
     if h.hexdigest() != NCU_TRAFFIC["sha1"]:

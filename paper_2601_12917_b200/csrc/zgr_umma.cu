@@ -13,7 +13,8 @@
 //       - U G is accumulated on top as  Ulo Ghi + Uhi Glo + Uhi Ghi  (bf16 split operands,
 //         about 2^-16 relative error per term), the strip of c b G living in shared memory as the
 //         K-major B operand for all row tiles of a work item.
-//   * The epilogue warps (one per 32 rows x 32 columns of a tile) read D with tcgen05.ld (one row per thread), add the isotropic
+//   * The epilogue warps, in two groups that take alternate tiles (32 rows x 64 columns per warp, 32 columns
+//     at a time), read D with tcgen05.ld (one row per thread), add the isotropic
 //     normals (Philox4x32-10 + Box-Muller in registers), round to the storage type and write the
 //     tile into the shared-memory buffer the TMA store reads.
 //
@@ -203,8 +204,9 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-// Tile configuration per contraction width.  TILE_N = 192 runs 24 epilogue warps on 128 x 192 tiles
-// (three 64-column boxes); TILE_N = 128 runs 16 on 128 x 128 tiles.
+// Tile configuration per contraction width: compile-time parameters (-D...) whose defaults are the measured
+// optimum on B200.  TILE_N = 192 runs 24 epilogue warps on 128 x 192 tiles (three 64-column boxes);
+// TILE_N = 128 runs 16 on 128 x 128 tiles.  S = theta stages, N = adjacent tiles per strip.
 #ifndef ZGR_TILE_N16
 #define ZGR_TILE_N16 128
 #endif
