@@ -9,7 +9,7 @@ perturb(+eps), perturb(-2 eps), restore_update(lr/Q) -- 3Q in-place sweeps over 
 `value` = model parameters stepped per second (parameters x steps / time, all ranks), measured with
 CUDA events with weights, subspaces and work tables resident in HBM.  `e2e` repeats the measurement
 with the per-step inputs coming from the host through the C ABI: every guided tensor's subspace is
-copied from pinned host memory (zgr_update_subspace), the step runs, and the per-tensor norms are read
+copied from pinned host memory (zgr_update_subspaces), the step runs, and the per-tensor norms are read
 back to the host (zgr_get_stats).  The weights themselves stay in HBM in both: keeping the model on
 the device and never materialising z is the point of the method.
 
@@ -322,8 +322,7 @@ def main():
         n_e2e = max(1, min(args.steps, 3))
 
         def e2e_step(t):
-            for l in guided:
-                z.update_subspace(l, host_U[l])
+            z.update_subspaces(guided, [host_U[l] for l in guided])
             run_step(z, wl, t, args.schedule)
             return z.get_stats(wl.seed(t, 0))
 

@@ -156,6 +156,14 @@ int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor);
  * ZGR_ESTATE: a perturbation is active. */
 int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_t src_is_host, void* stream);
 
+/* zgr_update_subspace for n tensors in one call (tensors[i] gets U_src[i]; U_src may be NULL, or hold NULL
+ * entries, for buffers already rewritten in place; all sources on the host or all on the device).  The copies are
+ * enqueued one by one; when the list names every tensor that the tensor-core path serves, their operand copies
+ * are rebuilt by a single launch instead of one per tensor, which is what a guided round that refreshes the
+ * whole model wants.  tensors: HOST array of pairwise different indices.  Errors as zgr_update_subspace, plus
+ * ZGR_EINVAL for n < 1 or a repeated index. */
+int zgr_update_subspaces(zgr_ctx* ctx, int32_t n, const int32_t* tensors, const float* const* U_src, int32_t src_is_host, void* stream);
+
 /* Norm bookkeeping for the adaptive choice of alpha mentioned in Sec. 1: for each tensor l,
  * out[3l+0] = sum (a Z_l)^2, out[3l+1] = sum (b U_l G_l)^2, out[3l+2] = sum z_l^2 for `seed`.
  * Reads no weights.  `out` is a HOST array of 3*n doubles; the call synchronises `stream`. */

@@ -51,6 +51,8 @@ struct zgr_ctx {
   std::map<uint64_t, double> ledger;  // seeds whose perturbation is applied to the weights -> sum of the coefficients applied
   uint64_t last_seed = 0;             // most recently swept seed (introspection)
   bool guided_at_init = false;        // b != 0 when the sweep plan was made
+  SplitJob* d_split_jobs = nullptr;   // one job per tensor served by the tcgen05 kernel: rebuild of its operand copy of U
+  int n_split_jobs = 0;
   std::vector<char> frag_stale;       // per tensor: the fragment-order copy of U (legacy tensor-core kernel) lags behind U
   std::vector<Group> groups_multi;    // plan of multi-seed sweeps when it differs from `groups` (legacy tensor-core path only)
   bool multi_planned = false;
@@ -437,6 +439,16 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
       }
     }
   }
+  if (rc == ZGR_OK) {
+    std::vector<SplitJob> jobs;
+    for (const TensorDesc& td : ctx->descs)
+      if (td.umma) jobs.push_back(SplitJob{td.U, td.Uhi, td.Ulo, td.rows, ((td.rows + 127) / 128) * 128, td.rank, td.kpad});
+    ctx->n_split_jobs = static_cast<int>(jobs.size());
+    if (!jobs.empty()) {
+      rc = dev_alloc(ctx, &ctx->d_split_jobs, jobs.size());
+      if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(ctx->d_split_jobs, jobs.data(), jobs.size() * sizeof(SplitJob), cudaMemcpyHostToDevice));
+    }
+  }
   if (rc == ZGR_OK) rc = dev_alloc(ctx, &ctx->d_tmaps, ctx->tmaps.size());
   if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(ctx->d_tmaps, ctx->tmaps.data(), ctx->tmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
   if (rc == ZGR_OK) rc = dev_alloc(ctx, &ctx->d_err, 1);
@@ -744,6 +756,55 @@ int zgr_debug_plan(const zgr_tensor* tensors, int32_t n, const zgr_config* cfg, 
       ++count;
     }
   *n_items = count;
+  return ZGR_OK;
+}
+
+int zgr_update_subspaces(zgr_ctx* ctx, int32_t n, const int32_t* tensors, const float* const* U_src, int32_t src_is_host, void* stream) {
+  if (!ctx || !tensors || n < 1) return ZGR_EINVAL;
+  std::vector<char> seen(ctx->descs.size(), 0);
+  int n_umma = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    const int32_t l = tensors[i];
+    if (l < 0 || l >= static_cast<int32_t>(ctx->descs.size()) || seen[static_cast<size_t>(l)]) return ZGR_EINVAL;
+    seen[static_cast<size_t>(l)] = 1;
+    if (ctx->descs[static_cast<size_t>(l)].rank == 0) return ZGR_EINVAL;
+    n_umma += ctx->descs[static_cast<size_t>(l)].umma ? 1 : 0;
+  }
+  if (ctx->sticky) return ctx->sticky;
+  if (!ctx->ledger.empty()) return ZGR_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // every tensor of the tcgen05 path is listed: their operand copies are rebuilt by one launch after the copies
+  const bool fused = n_umma > 0 && n_umma == ctx->n_split_jobs;
+  for (int32_t i = 0; i < n; ++i) {
+    const int32_t l = tensors[i];
+    TensorDesc& td = ctx->descs[static_cast<size_t>(l)];
+    const float* src = U_src ? U_src[i] : nullptr;
+    if (src != nullptr && src != td.U) {
+      const size_t bytes = static_cast<size_t>(td.rows) * td.rank * sizeof(float);
+      const int rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.U), src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, st));
+      if (rc != ZGR_OK) return rc;
+    }
+    if (td.Ufrag != nullptr) {
+      if (td.umma) {
+        ctx->frag_stale[static_cast<size_t>(l)] = 1;
+      } else {
+        const int rc = check(ctx, launch_split_subspace(td.U, td.rows, td.rank, td.kpad, const_cast<uint4*>(td.Ufrag), st));
+        if (rc != ZGR_OK) return rc;
+        ctx->launches++;
+      }
+    }
+    if (td.umma && !fused) {
+      const int64_t rows_pad = ((td.rows + 127) / 128) * 128;
+      const int rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.Uhi, td.Ulo, st));
+      if (rc != ZGR_OK) return rc;
+      ctx->launches++;
+    }
+  }
+  if (fused) {
+    const int rc = check(ctx, launch_split_subspace_rowmajor_all(ctx->d_split_jobs, ctx->n_split_jobs, st));
+    if (rc != ZGR_OK) return rc;
+    ctx->launches++;
+  }
   return ZGR_OK;
 }
 

@@ -32,6 +32,15 @@ size_t umma_smem_bytes(int kpad);
 cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
 cudaError_t launch_stats_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
 cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st);
+// The same for a device-resident list of tensors in one launch (grid.y = job).
+struct SplitJob {
+  const float* U;
+  void* hi;
+  void* lo;
+  int64_t rows, rows_pad;
+  int32_t r, kp;
+};
+cudaError_t launch_split_subspace_rowmajor_all(const SplitJob* d_jobs, int n_jobs, cudaStream_t st);
 
 cudaError_t launch_stats(int bits, const SweepParams& p, int grid, cudaStream_t st);
 cudaError_t launch_split_subspace(const float* U, int64_t rows, int r, int kp, uint4* out, cudaStream_t st);

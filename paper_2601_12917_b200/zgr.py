@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.zgr_get_scalars.argtypes = [vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
         L.zgr_get_state.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(u64), ctypes.POINTER(dbl)]
         L.zgr_update_subspace.argtypes = [vp, i32, vp, i32, vp]
+        L.zgr_update_subspaces.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(vp), i32, vp]
+        L.zgr_update_subspaces.restype = ctypes.c_int
         L.zgr_profile.argtypes = [vp, i32]
         L.zgr_profile_read.argtypes = [vp, ctypes.POINTER(ZgrKernelTime), i32, ctypes.POINTER(i32)]
         L.zgr_tensor_norms_noalloc.argtypes = [vp, u64, i32, vp, vp]
@@ -186,6 +188,24 @@ class Zgr:
             assert U_src.is_contiguous() and U_src.dtype == self._keep[1][tensor].dtype and U_src.shape == self._keep[1][tensor].shape
             ptr, host = U_src.data_ptr(), 0 if U_src.is_cuda else 1
         _check(lib().zgr_update_subspace(self._h, tensor, ptr, host, _stream_ptr(stream)), "zgr_update_subspace")
+
+    def update_subspaces(self, tensors: Sequence[int], U_srcs: Sequence, stream=None) -> None:
+        """New subspaces for several tensors in one call (zgr_update_subspaces); all sources on the host
+        (pinned for asynchronous copies) or all on the device, None for a buffer rewritten in place."""
+        n = len(tensors)
+        assert n == len(U_srcs) and n > 0
+        host = None
+        ptrs = (ctypes.c_void_p * n)()
+        for i, (l, U) in enumerate(zip(tensors, U_srcs)):
+            if U is None:
+                ptrs[i] = None
+                continue
+            assert U.is_contiguous() and U.dtype == self._keep[1][l].dtype and U.shape == self._keep[1][l].shape
+            assert host is None or host == (not U.is_cuda), "sources must be all on the host or all on the device"
+            host = not U.is_cuda
+            ptrs[i] = U.data_ptr()
+        _check(lib().zgr_update_subspaces(self._h, n, (ctypes.c_int32 * n)(*tensors), ptrs, 1 if host else 0, _stream_ptr(stream)),
+               "zgr_update_subspaces")
 
     def profile(self, enable: bool) -> None:
         _check(lib().zgr_profile(self._h, 1 if enable else 0), "zgr_profile")

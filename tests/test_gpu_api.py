@@ -121,3 +121,36 @@ def test_set_alpha_between_steps():
         q.lib.set_alpha(0.5)
     assert e.value.code == zgr.ESTATE
     q.lib.set_alpha(1.0)
+
+
+def test_update_subspaces_in_one_call():
+    """zgr_update_subspaces: all guided tensors at once (one fused rebuild of the operand copies), a subset
+    (per-tensor rebuilds), device and host sources, then argument errors."""
+    shapes, ranks = [(256, 384), (1, 40), (200, 512), (96, 256)], [32, 0, 16, 8]
+    p = Pair(shapes, ranks, "bf16", seed=9, bits=16)
+    p.step(seed=1, lp=2.0, lm=1.9, lr=1e-4)
+    new = {l: synth.subspace(shapes[l][0], ranks[l], 500 + l) for l in (0, 2, 3)}
+    launches0 = p.lib.launch_count()
+    p.lib.update_subspaces([0, 2, 3], [torch.from_numpy(new[l]).pin_memory() for l in (0, 2, 3)])      # whole model, host
+    assert p.lib.launch_count() - launches0 == 1                  # one fused launch for the two tensor-core tensors; rank 8 reads U directly
+    torch.cuda.synchronize()
+    for l in (0, 2, 3):
+        np.testing.assert_array_equal(p.U[l].cpu().numpy(), new[l])
+    reports = p.step(seed=2, lp=1.7, lm=2.2, lr=1e-4)
+    assert min(rep["moved"] for call in reports for rep in call) > 0.3
+    newer = synth.subspace(200, 16, 777)
+    p.lib.update_subspaces([2], [torch.from_numpy(newer).cuda()])                                      # subset, device
+    p.step(seed=3, lp=2.1, lm=2.0, lr=1e-4)
+    p.U[0].copy_(torch.from_numpy(synth.subspace(256, 32, 778)))
+    p.lib.update_subspaces([0, 2], [None, None])                                                       # rewritten in place
+    p.step(seed=4, lp=2.1, lm=2.0, lr=1e-4)
+    for bad in ([], [1], [0, 0], [9]):
+        with pytest.raises((zgr.ZgrError, AssertionError)) as e:
+            p.lib.update_subspaces(bad, [None] * len(bad))
+        if isinstance(e.value, zgr.ZgrError):
+            assert e.value.code == zgr.EINVAL
+    p.lib.perturb(5, 1e-3)
+    with pytest.raises(zgr.ZgrError) as e:
+        p.lib.update_subspaces([0], [None])
+    assert e.value.code == zgr.ESTATE
+    p.lib.restore_update(5, 2.0, 2.0, 0.0)
