@@ -311,6 +311,13 @@ def main():
                     "peak_kind": f"of {peak_kind}", "kernel": kname, "launches": top["launches"],
                     "ms_per_launch": per_launch_ms, "algorithmic_bytes_per_launch": 2 * eb * top["elements"],
                     "share_of_kernel_time": top["ms_total"] / sum(k["ms_total"] for k in kernels)}
+        # second bound of the same kernel: the special-function pipe that the Gaussian transform runs on.
+        # 16 lanes per clock per SM x 148 SMs x 1.965 GHz; the transform costs four operations per pair of
+        # normals (lg2, sqrt, sin, cos), i.e. 2 per element, in both generator modes.
+        sfu_peak = 16 * 148 * 1.965e9 / 2.0
+        roofline["sfu"] = {"bound": "alu", "achieved": top["elements"] / (per_launch_ms * 1e-3), "peak": sfu_peak,
+                           "unit": "elements/s", "frac": top["elements"] / (per_launch_ms * 1e-3) / sfu_peak,
+                           "peak_kind": "nominal: 16 special-function lanes/clk/SM x 148 SMs x 1.965 GHz / 2 operations per element"}
 
     # ---- end to end: per-step inputs from pinned host memory, result read back ----
     e2e = None
