@@ -39,7 +39,7 @@ UNIT = "params/s"
 NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.76e9,
                "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
                            "paper_2601_12917_b200/csrc/zgr_internal.h"],
-               "sha1": "34e2c55264b480439074b4fc8f445f816e3226fe"}
+               "sha1": "cac5ba61094e317b1df2c4a422e189a3f4b943ff"}
 
 
 def _code_only(text: str) -> str:

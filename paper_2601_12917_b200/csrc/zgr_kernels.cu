@@ -405,6 +405,35 @@ __global__ void split_subspace_kernel(const float* __restrict__ U, int64_t rows,
   out[idx] = make_uint4(regs[0], regs[1], regs[2], regs[3]);
 }
 
+// U (rows x r fp32) -> two row-major bf16 matrices (hi, lo), rows padded to a multiple of 128 and
+// columns to KP with zeros: the TMA source of the A operand.
+__global__ void split_subspace_rowmajor_kernel(const float* __restrict__ U, int64_t rows, int r, int kp, int64_t rows_pad,
+                                               __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+  if (idx >= rows_pad * kp) return;
+  const int64_t row = idx / kp;
+  const int k = static_cast<int>(idx % kp);
+  const float x = (row < rows && k < r) ? U[row * r + k] : 0.0f;
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  hi[idx] = h;
+  lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+__global__ void split_subspace_rowmajor_all_kernel(const SplitJob* __restrict__ jobs) {
+  const SplitJob j = jobs[blockIdx.y];
+  const int64_t n = j.rows_pad * j.kp;
+  __nv_bfloat16* hi = static_cast<__nv_bfloat16*>(j.hi);
+  __nv_bfloat16* lo = static_cast<__nv_bfloat16*>(j.lo);
+  for (int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; idx < n; idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t row = idx / j.kp;
+    const int k = static_cast<int>(idx % j.kp);
+    const float x = (row < j.rows && k < j.r) ? j.U[row * j.r + k] : 0.0f;
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    hi[idx] = h;
+    lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
+  }
+}
+
 // Raw generator blocks (test hook).
 __global__ void philox_blocks_kernel(PhiloxKeys keys, uint32_t tensor, uint32_t tag, uint64_t first_block, int64_t n_blocks,
                                      uint32_t* __restrict__ out) {
@@ -509,6 +538,20 @@ cudaError_t launch_split_subspace(const float* U, int64_t rows, int r, int kp, u
   const int block = 256;
   const int64_t grid = (n_out + block - 1) / block;
   split_subspace_kernel<<<static_cast<unsigned>(grid), block, 0, st>>>(U, rows, r, kp, out, n_out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split_subspace_rowmajor_all(const SplitJob* d_jobs, int n_jobs, cudaStream_t st) {
+  if (n_jobs <= 0) return cudaSuccess;
+  split_subspace_rowmajor_all_kernel<<<dim3(64, static_cast<unsigned>(n_jobs)), 256, 0, st>>>(d_jobs);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st) {
+  const int64_t n = rows_pad * kp;
+  const int block = 256;
+  split_subspace_rowmajor_kernel<<<static_cast<unsigned>((n + block - 1) / block), block, 0, st>>>(
+      U, rows, r, kp, rows_pad, static_cast<__nv_bfloat16*>(hi), static_cast<__nv_bfloat16*>(lo));
   return cudaGetLastError();
 }
 

@@ -637,35 +637,6 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
   }
 }
 
-// U (rows x r fp32) -> two row-major bf16 matrices (hi, lo), rows padded to a multiple of 128 and
-// columns to KP with zeros: the TMA source of the A operand.
-__global__ void split_subspace_rowmajor_kernel(const float* __restrict__ U, int64_t rows, int r, int kp, int64_t rows_pad,
-                                               __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
-  const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
-  if (idx >= rows_pad * kp) return;
-  const int64_t row = idx / kp;
-  const int k = static_cast<int>(idx % kp);
-  const float x = (row < rows && k < r) ? U[row * r + k] : 0.0f;
-  const __nv_bfloat16 h = __float2bfloat16_rn(x);
-  hi[idx] = h;
-  lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
-}
-
-__global__ void split_subspace_rowmajor_all_kernel(const SplitJob* __restrict__ jobs) {
-  const SplitJob j = jobs[blockIdx.y];
-  const int64_t n = j.rows_pad * j.kp;
-  __nv_bfloat16* hi = static_cast<__nv_bfloat16*>(j.hi);
-  __nv_bfloat16* lo = static_cast<__nv_bfloat16*>(j.lo);
-  for (int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; idx < n; idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-    const int64_t row = idx / j.kp;
-    const int k = static_cast<int>(idx % j.kp);
-    const float x = (row < j.rows && k < j.r) ? j.U[row * j.r + k] : 0.0f;
-    const __nv_bfloat16 h = __float2bfloat16_rn(x);
-    hi[idx] = h;
-    lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
-  }
-}
-
 size_t umma_smem_bytes(int kpad) {
   return kpad == 16 ? UmmaCfg<16>::SMEM_BYTES : (kpad == 32 ? UmmaCfg<32>::SMEM_BYTES : UmmaCfg<64>::SMEM_BYTES);
 }
@@ -710,20 +681,6 @@ cudaError_t launch_stats_umma(const KernelChoice& kc, const SweepParams& p, cons
   // the storage type plays no role when no weights are touched: one instantiation serves all
   return kc.bits == 32 ? launch_umma_kp<__nv_bfloat16, 32, true>(kc.kpad, p, tmaps, error, grid, st)
                        : launch_umma_kp<__nv_bfloat16, 16, true>(kc.kpad, p, tmaps, error, grid, st);
-}
-
-cudaError_t launch_split_subspace_rowmajor_all(const SplitJob* d_jobs, int n_jobs, cudaStream_t st) {
-  if (n_jobs <= 0) return cudaSuccess;
-  split_subspace_rowmajor_all_kernel<<<dim3(64, static_cast<unsigned>(n_jobs)), 256, 0, st>>>(d_jobs);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st) {
-  const int64_t n = rows_pad * kp;
-  const int block = 256;
-  split_subspace_rowmajor_kernel<<<static_cast<unsigned>((n + block - 1) / block), block, 0, st>>>(
-      U, rows, r, kp, rows_pad, static_cast<__nv_bfloat16*>(hi), static_cast<__nv_bfloat16*>(lo));
-  return cudaGetLastError();
 }
 
 }  // namespace zgr
