@@ -36,10 +36,10 @@ UNIT = "params/s"
 
 # DRAM traffic per launch of the dominant kernel from one ncu capture (profiles/sweep_umma_bf16_k32_llama7b.md:
 # small case, scaled by the elements processed), valid only for the kernel sources it was taken from.
-NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.76e9,
+NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.77e9,
                "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
                            "paper_2601_12917_b200/csrc/zgr_internal.h"],
-               "sha1": "cac5ba61094e317b1df2c4a422e189a3f4b943ff"}
+               "sha1": "e554e3bd71448c7b4aba5b241ad4648c1002e874"}
 
 
 def _code_only(text: str) -> str:
