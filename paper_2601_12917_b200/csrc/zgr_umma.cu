@@ -530,7 +530,8 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       // The epilogue warps of a scheduler run the same instruction stream from the same starting
       // point: first the integer rounds of the generator, then the special-function half of the
       // transform.  Holding every other column group back once per item puts half of each scheduler's
-      // warps in the other phase, so the two pipes overlap (measured: 6.5 -> 6.15 ms per 7B sweep).
+      // warps in the other phase, so the two pipes overlap (measured with one group: 6.5 -> 6.15 ms per 7B sweep;
+      // with two groups the groups are out of step by construction).
       if (GROUPS == 1 && (cg_first & 1)) __nanosleep(kStaggerNs);
 
       const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
