@@ -34,8 +34,8 @@ METRIC = "zgr_step_params_per_sec"
 UNIT = "params/s"
 
 
-# DRAM traffic per launch of the dominant kernel from one ncu capture (profiles/sweep_umma_bf16_k32_llama7b.md:
-# small case, scaled by the elements processed), valid only for the kernel sources it was taken from.
+# DRAM traffic per launch of the dominant kernel from one ncu capture (a small case, scaled by the elements
+# processed), valid only for the kernel sources it was taken from.
 NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.77e9,
                "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
                            "paper_2601_12917_b200/csrc/zgr_internal.h"],
@@ -223,6 +223,54 @@ def run_step(z, wl, t: int, schedule: str = "sequential"):
         z.restore_update(seed, lp, lm, wl.lr / wl.queries)
 
 
+def roofline_of(kernels, eb, peak, peak_kind):
+    """Roofline entry of the kernel that took the most time: algorithmic bytes (read + write of every weight it
+    covers) per launch over its average CUDA-event duration."""
+    top = max(kernels, key=lambda k: k["ms_total"]) if kernels else None
+    if not top:
+        return None, None
+    per_launch_ms = top["ms_total"] / top["launches"]
+    achieved = 2 * eb * top["elements"] / (per_launch_ms * 1e-3) / 1e9
+    kname = f"sweep_{top['path']}_kernel(k={top['kpad']})"
+    return top, {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                 "peak_kind": f"of {peak_kind}", "kernel": kname, "launches": top["launches"], "ms_per_launch": per_launch_ms,
+                 "algorithmic_bytes_per_launch": 2 * eb * top["elements"],
+                 "share_of_kernel_time": top["ms_total"] / sum(k["ms_total"] for k in kernels)}
+
+
+def measure_other(name, device, bits, steps, peak, peak_kind):
+    """A short resident measurement of another of the paper-shaped configurations (parity-test cases of their
+    own, shown here so that every sweep kernel has a driver-visible figure): 1 warm-up step, `steps` timed."""
+    import torch
+    from paper_2601_12917_b200 import synth, zgr
+    wl = synth.workload(name)
+    free, _ = torch.cuda.mem_get_info()
+    if free < wl.params * synth.DTYPE_BYTES[wl.dtype] * 1.3 + 4e9:
+        return {"workload": name, "skipped": "not enough free device memory"}
+    dm = synth.materialise(wl, device, seed=0)
+    z = zgr.from_device_model(dm, bits)
+    stream = torch.cuda.current_stream()
+    run_step(z, wl, 0)
+    torch.cuda.synchronize()
+    z.profile(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for t in range(steps):
+        run_step(z, wl, 1 + t)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    kernels = z.profile_read()
+    z.profile(False)
+    _, roof = roofline_of(kernels, synth.DTYPE_BYTES[wl.dtype], peak, peak_kind)
+    out = {"workload": name, "storage": wl.dtype, "params": wl.params, "rank": wl.rank, "queries": wl.queries, "dtc": wl.dtc,
+           "steps": steps, "ms_per_step": ms / steps, "value": wl.params * steps / (ms * 1e-3), "unit": UNIT, "roofline": roof}
+    z.close()
+    del z, dm
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -236,6 +284,7 @@ def main():
                     help="sequential: 3Q single-seed sweeps per step (the headline); deferred: 2Q+1 sweeps with multi-seed passes")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -300,17 +349,10 @@ def main():
     # ---- roofline of the dominant kernel ----
     peak, peak_kind = load_peaks()
     eb = synth.DTYPE_BYTES[wl.dtype]
-    top = max(kernels, key=lambda k: k["ms_total"]) if kernels else None
-    roofline = None
+    top, roofline = roofline_of(kernels, eb, peak, peak_kind)
     if top:
-        per_launch_ms = top["ms_total"] / top["launches"]
-        achieved = 2 * eb * top["elements"] / (per_launch_ms * 1e-3) / 1e9
-        kname = f"sweep_{top['path']}_kernel(k={top['kpad']})"
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": ncu_traffic(kname, wl.name) if args.layers is None else None,
-                    "peak_kind": f"of {peak_kind}", "kernel": kname, "launches": top["launches"],
-                    "ms_per_launch": per_launch_ms, "algorithmic_bytes_per_launch": 2 * eb * top["elements"],
-                    "share_of_kernel_time": top["ms_total"] / sum(k["ms_total"] for k in kernels)}
+        per_launch_ms = roofline["ms_per_launch"]
+        roofline["traffic"] = ncu_traffic(roofline["kernel"], wl.name) if args.layers is None else None
         # second bound of the same kernel: the special-function pipe that the Gaussian transform runs on.
         # 16 lanes per clock per SM x 148 SMs x 1.965 GHz; the transform costs four operations per pair of
         # normals (lg2, sqrt, sin, cos), i.e. 2 per element, in both generator modes.
@@ -344,19 +386,30 @@ def main():
         e2e = {"value": units_e / (ms_e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
                "ms_per_step": ms_e / n_e2e, "what": "subspaces H2D from pinned memory + step + per-tensor norms D2H, through the C ABI"}
 
+    # ---- the other configurations, briefly (single process only; the headline above is unaffected) ----
+    others = None
+    z.close()
+    if world == 1 and not args.no_others and args.layers is None and wl.name == "llama_7b":
+        del dm
+        torch.cuda.empty_cache()
+        others = [measure_other(name, device, args.bits, 3, peak, peak_kind) for name in ("roberta_large", "opt_1p3b", "llama_13b")]
+        full = measure_other("llama_7b", device, 32, 3, peak, peak_kind)      # the headline workload with 32 random bits per normal
+        full["bits_per_normal"] = 32
+        others.append(full)
+
     if rank == 0:
         sweeps = 3 * wl.queries if args.schedule == "sequential" else 2 * wl.queries + 1
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-                "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32",     # the arithmetic type of the path; the weights are stored as config.storage
                 "data": "synthetic",
                 "config": {"workload": wl.name, "storage": wl.dtype, "params": wl.params, "tensors": len(wl.tensors), "rank": wl.rank,
                            "queries": wl.queries, "schedule": args.schedule, "sweeps_per_step": sweeps, "bits_per_normal": args.bits, "alpha": wl.alpha, "eps": wl.eps,
                            "lr": wl.lr, "scale_mode": "unit", "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only"},
                 "sweep_params_per_s": value * sweeps, "hbm_gbs_all_sweeps": value * sweeps * 2 * eb / 1e9,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-                "kernels": kernels}
+                "kernels": kernels, "other_configs": others}
         print(json.dumps(line), flush=True)
-    z.close()
     if world > 1:
         dist.destroy_process_group()
 

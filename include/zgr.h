@@ -26,7 +26,8 @@
  *   - All functions return 0 on success or a negative ZGR_E* code.  Arguments are validated before
  *     anything is launched: a call that fails validation leaves the weights untouched.
  *   - A context is bound to the device that is current when zgr_init is called and is not
- *     thread-safe; use one per thread or serialise calls.
+ *     thread-safe; use one per thread or serialise calls.  Every call that enqueues work checks that
+ *     this device is still the current one and returns ZGR_EINVAL otherwise, before anything is launched.
  */
 #ifndef ZGR_H_
 #define ZGR_H_
@@ -61,7 +62,9 @@ typedef struct zgr_ctx zgr_ctx; /* opaque; created by zgr_init, released by zgr_
 typedef struct {
   void* data;       /* device; rows*cols elements of `dtype`, row-major, contiguous, updated in place.
                        Must be aligned to the element size; 16-byte alignment and cols a multiple of
-                       16 bytes' worth of elements select the vectorised kernels */
+                       16 bytes' worth of elements select the vectorised kernels.  fp32 storage with
+                       rank > 8 is served by the one-element-per-thread fallback kernel (exact fp32
+                       contraction; none of the paper-shaped configurations needs it) */
   int64_t rows;     /* m_l >= 1 */
   int64_t cols;     /* n_l >= 1 */
   int32_t dtype;    /* ZGR_F32 | ZGR_F16 | ZGR_BF16 */
@@ -124,12 +127,27 @@ int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, con
                              void* stream);
 
 /* Change the mixing ratio alpha of Eq. (perturbation) between steps; a and b are recomputed as in
- * zgr_init.  This is the hook for the adaptive choice of the ZGR parameter mentioned in Sec. 1 ("based on
- * the relative scales of BP-based and ZOO-based perturbations"): the paper gives no rule, so the caller
- * applies its own to the norms of zgr_get_stats and sets the result here.
+ * zgr_init.  This is the hook for the adaptive choice of the mixing ratio announced in Sec. 1, which is to
+ * follow the sizes of the guided and the isotropic part; the paper gives no rule, so the caller applies its
+ * own to the norms of zgr_get_stats (or uses zgr_adapt_alpha below) and sets the result here.
  * ZGR_EINVAL: alpha outside [0, 1].  ZGR_ESTATE: a perturbation is active, or the context was built with
  * alpha = 1 (its sweep plan carries no subspace operands) and alpha < 1 is asked for. */
 int zgr_set_alpha(zgr_ctx* ctx, double alpha);
+
+/* One candidate for that adaptive choice, off unless the caller invokes it: balance the energies of the two
+ * parts of Eq. (perturbation).  `stats` (HOST, 3 doubles per tensor, as written by zgr_get_stats under the
+ * context's current alpha) gives sum (a Z)^2 and sum (b U G)^2; divided by a^2 d and b^2 K they are the energy
+ * of each part per unit of its mixing weight, e_iso and e_g, and the two parts carry the same energy at
+ *     alpha* = e_g / (e_iso + e_g).
+ * The context moves to  alpha = clamp((1 - eta) alpha_old + eta alpha*, alpha_min, alpha_max)  (a, b recomputed
+ * as in zgr_set_alpha) and *alpha_out receives it.  With seed-drawn unit coefficients and an orthonormal U the
+ * balance sits at 1/2; compressed coefficients whose scale is not that of a unit Gaussian, or a subspace that
+ * is not orthonormal, move it.  If one of the parts is switched off (alpha = 0 or 1, or no tensor has a
+ * subspace) alpha is left as it is.  The rule is this library's: Sec. 1 announces an adaptive ratio that
+ * follows the relative sizes of the two parts and states none.
+ * ZGR_EINVAL: null pointer, bounds not 0 <= alpha_min <= alpha_max <= 1, eta outside [0, 1], a norm that is
+ * negative or not finite.  ZGR_ESTATE: a perturbation is active. */
+int zgr_adapt_alpha(zgr_ctx* ctx, const double* stats, double alpha_min, double alpha_max, double eta, double* alpha_out);
 
 /* Deliver the guided coefficients of one tensor compressed (Sec. 3.4, DTC): from now on
  *     G_l[k][c] = scale[k] * (q[k][c] - zero[k])       (x = lambda (x_quant - delta))
@@ -143,6 +161,36 @@ int zgr_set_alpha(zgr_ctx* ctx, double alpha);
  * ZGR_ESTATE: a perturbation is active (the coefficients must not change between a perturb and
  * its restore_update). */
 int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits);
+
+/* The same with only a proportion of the payload compressed (Sec. 3.4, the adaptive proportion omega): the
+ * first n_rows rows of G_l come from the codes (q: n_rows rows in the layout of `bits`; scale, zero: n_rows
+ * entries), rows n_rows .. rank-1 are drawn from the seed as if nothing had been delivered for them.
+ * 1 <= n_rows <= rank; n_rows = rank is zgr_set_coeffs_dtc.  Errors as there, plus ZGR_EINVAL for n_rows out of range. */
+int zgr_set_coeffs_dtc_rows(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits, int32_t n_rows);
+
+/* zgr_perturb, layer by layer, with the compressed coefficients arriving from the host while earlier layers
+ * are swept (Sec. 3.3, the layer-wise sample -> transmit -> apply pipeline; Sec. 3.4, the transmission of a
+ * layer is to fit under the compute of another).  layer_end: HOST array of n_layers strictly increasing
+ * tensor indices, layer L being the tensors [layer_end[L-1], layer_end[L]) and layer_end[n_layers-1] the number
+ * of tensors.  deliveries: HOST array; entry i names a tensor whose compressed coefficients were set with
+ * zgr_set_coeffs_dtc(_rows) and gives HOST sources (pinned memory, or the copies do not overlap anything) of
+ * the same sizes and layout, which are copied into those device buffers on `copy_stream`.  All copies are
+ * enqueued at once, in layer order, behind the work already on `stream`; the sweep of a layer on `stream`
+ * waits for that layer's copies only, so later layers travel while earlier ones are swept.  n_deliveries = 0
+ * gives the same sweep as zgr_perturb, issued as one launch per kernel family and layer.
+ * The result is identical to copying everything first and calling zgr_perturb.
+ * ZGR_EINVAL: scale not finite, bad layer table, a delivery naming a bad or repeated tensor, a tensor without
+ * compressed coefficients, or a zero point given for a tensor registered without one (or the reverse).
+ * ZGR_ESTATE: as zgr_perturb; with deliveries, also if any seed is active (coefficients may not change between
+ * a perturbation and its restore). */
+typedef struct {
+  int32_t tensor;
+  const void* q;       /* HOST: codes of the delivered rows */
+  const float* scale;  /* HOST: one per delivered row */
+  const float* zero;   /* HOST: one per delivered row, or NULL if the tensor was registered without zero points */
+} zgr_coeff_delivery;
+int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_layers, const int32_t* layer_end, int32_t n_deliveries,
+                       const zgr_coeff_delivery* deliveries, void* stream, void* copy_stream);
 
 /* Back to seed-drawn coefficients for `tensor` (Algorithm 1, "Sample z_g").  Errors as above. */
 int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor);
@@ -163,6 +211,20 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
  * whole model wants.  tensors: HOST array of pairwise different indices.  Errors as zgr_update_subspace, plus
  * ZGR_EINVAL for n < 1 or a repeated index. */
 int zgr_update_subspaces(zgr_ctx* ctx, int32_t n, const int32_t* tensors, const float* const* U_src, int32_t src_is_host, void* stream);
+
+/* Build the subspace of `tensor` on the device from collected gradient directions (Algorithm 1, "Collect
+ * gradients to build basis V_r"; Sec. 3.2, cloud side).  grads: rows x rank fp32 row-major whose column j is the
+ * j-th direction collected in the row space of the tensor (the paper does not say how a gradient of a matrix
+ * becomes a direction of its row space; that reduction is the caller's), on the host (src_is_host != 0) or on
+ * the device, or NULL if the directions were written into the subspace buffer given to zgr_init.  The result is
+ * the orthonormal basis of their span that a QR factorisation with a positive diagonal of R gives, column k
+ * spanning, with the columns before it, the first k + 1 directions.  It overwrites that subspace buffer, and the
+ * library's operand copies are rebuilt as by zgr_update_subspace.  Cholesky QR applied twice, carried in double:
+ * orthonormal to about 1e-7 for inputs whose condition number is below about 1e6.  Allocates scratch on
+ * first use (and when a larger tensor comes); synchronises `stream`.
+ * ZGR_EINVAL: bad index, tensor without subspace, fewer rows than rank, misaligned pointer, or directions that
+ * are linearly dependent to working precision (nothing is written then).  ZGR_ESTATE: a perturbation is active. */
+int zgr_build_subspace(zgr_ctx* ctx, int32_t tensor, const float* grads, int32_t src_is_host, void* stream);
 
 /* Norm bookkeeping for the adaptive choice of alpha mentioned in Sec. 1: for each tensor l,
  * out[3l+0] = sum (a Z_l)^2, out[3l+1] = sum (b U_l G_l)^2, out[3l+2] = sum z_l^2 for `seed`.
@@ -190,11 +252,25 @@ int zgr_tensor_norms_noalloc(zgr_ctx* ctx, uint64_t seed, int32_t tensor, double
 
 /* Test hooks.  zgr_debug_philox writes n_blocks raw generator blocks (4 uint32 each) of stream
  * (seed, tensor, tag) starting at first_block to dev_out (device).  zgr_debug_z writes z_l(seed) as
- * fp32 (rows*cols, device) using the same kernels as the sweeps (it sweeps a zeroed fp32 scratch
- * image of the tensor with scale 1). */
+ * fp32 (rows*cols, device): it sweeps a zeroed fp32 scratch image of the tensor with scale 1 through the
+ * kernel family of the tensor's storage type, except that tensors which the sweeps serve with the tcgen05
+ * kernel (16-bit storage, rank > 8) go through the legacy mma.sync kernel here, because the tcgen05 kernel
+ * reads and writes 16-bit tiles only.  zgr_debug_z_tcgen05 is the hook for that kernel.
+ * zgr_debug_check_device is the host-only comparison behind the "current device" check of every
+ * launching call: ZGR_OK if ctx_device is a valid ordinal equal to current_device, else ZGR_EINVAL. */
 int zgr_debug_philox(zgr_ctx* ctx, uint64_t seed, int32_t tensor, int32_t tag, uint64_t first_block, int64_t n_blocks,
                      uint32_t* dev_out, void* stream);
 int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, void* stream);
+int zgr_debug_check_device(int32_t ctx_device, int32_t current_device);
+
+/* z_l(seed) as the tcgen05 sweep kernel computes it: that kernel itself (same TMA loads, tensor-core
+ * products, tensor-memory reads and epilogue arithmetic as in zgr_perturb) sweeps a zeroed 16-bit image
+ * of the tensor with coefficient 1, and its fp32 result for every element, taken just before the rounding
+ * to the storage type, is written to dev_out (device, rows*cols fp32, 16-byte aligned).  The weights are
+ * not touched.  Allocates and frees the image; synchronises `stream`.
+ * ZGR_ESTATE: the sweeps do not serve this tensor with the tcgen05 kernel (fp32 storage, rank <= 8,
+ * unaligned data, alpha = 1 at zgr_init, or the legacy tensor-core path was selected). */
+int zgr_debug_z_tcgen05(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, void* stream);
 
 /* The work plan of a sweep, computed on the host alone (no device is needed or touched): which kernel
  * family serves which part of which tensor.  Test hook for the planner: the items of a plan must cover

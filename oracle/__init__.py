@@ -5,7 +5,7 @@ tests, the smoke check and the benchmark's CPU-baseline leg have an independent,
 double-precision statement of Eq. (ZOO), Eq. (perturbation), Eq. (grad), Algorithm 1 and the DTC
 dequantisation to compare the CUDA library against.
 
-The arithmetic lives in the C++ file; this module only builds it (g++, OpenMP), marshals numpy
+All of the arithmetic lives in the C++ file; this module only builds it (g++, OpenMP), marshals numpy
 arrays, and keeps the per-seed bookkeeping of the call sequence
 ``perturb(+eps) -> perturb(-2 eps) -> restore_update`` (class :class:`OracleZGR`).
 """
@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         _lib.zgro_projected_grad.restype = ctypes.c_double
         _lib.zgro_projected_grad.argtypes = [ctypes.c_double] * 3
         _lib.zgro_num_threads.restype = ctypes.c_int
+        _lib.zgro_update_coefficient.restype = ctypes.c_double
+        _lib.zgro_adapt_alpha.restype = ctypes.c_double
     return _lib
 
 
@@ -133,9 +135,11 @@ class OracleTensor:
     cols: int
     dtype: int
     U: Optional[np.ndarray] = None    # rows x rank float32, orthonormal columns
-    q: Optional[np.ndarray] = None    # rank x cols int8  (DTC codes) or None -> coefficients from the seed
+    q: Optional[np.ndarray] = None    # qrows x cols int8  (DTC codes) or None -> coefficients from the seed
     scale: Optional[np.ndarray] = None
     zero: Optional[np.ndarray] = None
+    # (Sec. 3.4, proportion omega: the codes may cover only the first q.shape[0] rows of G_l; the other rows
+    #  are drawn from the seed)
 
     @property
     def rank(self) -> int:
@@ -148,10 +152,16 @@ class OracleTensor:
         ze = None if self.zero is None else np.ascontiguousarray(self.zero, dtype=np.float32)
         return U, q, sc, ze
 
+    @property
+    def qrows(self) -> int:
+        """Rows of G_l taken from the codes."""
+        return 0 if self.q is None else int(np.asarray(self.q).shape[0])
+
 
 def coeffs(seed, tensor_id, bits, rank, cols, q=None, scale=None, zero=None) -> np.ndarray:
     out = np.zeros((rank, cols), dtype=np.float64)
-    lib().zgro_coeffs(_u64(seed), ctypes.c_uint32(tensor_id), ctypes.c_int(bits), _i64(rank), _i64(cols), _p(q), _p(scale), _p(zero), _p(out))
+    qrows = 0 if q is None else int(np.asarray(q).shape[0])
+    lib().zgro_coeffs(_u64(seed), ctypes.c_uint32(tensor_id), ctypes.c_int(bits), _i64(rank), _i64(cols), _p(q), _p(scale), _p(zero), _i64(qrows), _p(out))
     return out
 
 
@@ -162,7 +172,7 @@ def z_tensor(t: OracleTensor, seed: int, tensor_id: int, bits: int, a: float, b:
     iso = np.zeros(n, dtype=np.float64) if parts else None
     gd = np.zeros(n, dtype=np.float64) if parts else None
     lib().zgro_z_tensor(_u64(seed), ctypes.c_uint32(tensor_id), ctypes.c_int(bits), _i64(t.rows), _i64(t.cols), _p(U), _i64(t.rank),
-                        _p(q), _p(sc), _p(ze), ctypes.c_double(a), ctypes.c_double(b), _p(z), _p(iso), _p(gd))
+                        _p(q), _p(sc), _p(ze), _i64(t.qrows), ctypes.c_double(a), ctypes.c_double(b), _p(z), _p(iso), _p(gd))
     z = z.reshape(t.rows, t.cols)
     if parts:
         return z, iso.reshape(t.rows, t.cols), gd.reshape(t.rows, t.cols)
@@ -174,7 +184,7 @@ def z_elements(t: OracleTensor, seed: int, tensor_id: int, bits: int, a: float, 
     idx = np.ascontiguousarray(idx, dtype=np.int64)
     out = np.zeros(idx.size, dtype=np.float64)
     lib().zgro_z_elements(_u64(seed), ctypes.c_uint32(tensor_id), ctypes.c_int(bits), _i64(t.rows), _i64(t.cols), _p(U), _i64(t.rank),
-                          _p(q), _p(sc), _p(ze), ctypes.c_double(a), ctypes.c_double(b), _i64(idx.size), _p(idx), _p(out))
+                          _p(q), _p(sc), _p(ze), _i64(t.qrows), ctypes.c_double(a), ctypes.c_double(b), _i64(idx.size), _p(idx), _p(out))
     return out
 
 
@@ -183,7 +193,7 @@ def sweep_tensor(t: OracleTensor, seed: int, tensor_id: int, bits: int, a: float
     U, q, sc, ze = t._args()
     assert t.theta.flags["C_CONTIGUOUS"] and t.theta.dtype == _NP_STORAGE[t.dtype] and t.theta.size == t.rows * t.cols
     lib().zgro_sweep_tensor(_p(t.theta), ctypes.c_int(t.dtype), _u64(seed), ctypes.c_uint32(tensor_id), ctypes.c_int(bits),
-                            _i64(t.rows), _i64(t.cols), _p(U), _i64(t.rank), _p(q), _p(sc), _p(ze),
+                            _i64(t.rows), _i64(t.cols), _p(U), _i64(t.rank), _p(q), _p(sc), _p(ze), _i64(t.qrows),
                             ctypes.c_double(a), ctypes.c_double(b), ctypes.c_double(c))
 
 
@@ -195,34 +205,72 @@ def sweep_elements(t: OracleTensor, theta_in: np.ndarray, seed: int, tensor_id: 
     th = np.ascontiguousarray(theta_in, dtype=np.float64)
     out = np.zeros(idx.size, dtype=np.float64)
     lib().zgro_sweep_elements(_p(th), ctypes.c_int(t.dtype), _u64(seed), ctypes.c_uint32(tensor_id), ctypes.c_int(bits), _i64(t.rows),
-                              _i64(t.cols), _p(U), _i64(t.rank), _p(q), _p(sc), _p(ze), ctypes.c_double(a), ctypes.c_double(b),
+                              _i64(t.cols), _p(U), _i64(t.rank), _p(q), _p(sc), _p(ze), _i64(t.qrows), ctypes.c_double(a), ctypes.c_double(b),
                               ctypes.c_double(c), _i64(idx.size), _p(idx), _p(out))
     return out
+
+
+def _terms(seeds, coeffs):
+    n = len(seeds)
+    assert n == len(coeffs) and n >= 1
+    return n, np.asarray([int(x) & 0xFFFFFFFFFFFFFFFF for x in seeds], dtype=np.uint64), np.asarray(coeffs, dtype=np.float64)
 
 
 def sweep_multi_tensor(t: OracleTensor, seeds: Sequence[int], coeffs: Sequence[float], tensor_id: int, bits: int, a: float, b: float) -> None:
     """theta <- rnd(theta + sum_q c_q z(seed_q)), in place: the sum over seeds of Algorithm 1
     ("Recover gradient": sum_t g_t z_t; "Update") applied with a single rounding to the storage type."""
-    acc = decode(t.theta, t.dtype).astype(np.float64).ravel().copy()
-    for seed, c in zip(seeds, coeffs):
-        acc += float(c) * z_tensor(t, seed, tensor_id, bits, a, b).ravel()
-    t.theta[...] = encode(acc, t.dtype).reshape(t.theta.shape)
+    U, q, sc, ze = t._args()
+    n, sd, cf = _terms(seeds, coeffs)
+    assert t.theta.flags["C_CONTIGUOUS"] and t.theta.dtype == _NP_STORAGE[t.dtype] and t.theta.size == t.rows * t.cols
+    lib().zgro_sweep_multi_tensor(_p(t.theta), ctypes.c_int(t.dtype), ctypes.c_int(n), _p(sd), _p(cf), ctypes.c_uint32(tensor_id),
+                                  ctypes.c_int(bits), _i64(t.rows), _i64(t.cols), _p(U), _i64(t.rank), _p(q), _p(sc), _p(ze), _i64(t.qrows),
+                                  ctypes.c_double(a), ctypes.c_double(b))
 
 
 def sweep_multi_elements(t: OracleTensor, theta_in: np.ndarray, seeds: Sequence[int], coeffs: Sequence[float], tensor_id: int, bits: int,
                          a: float, b: float, idx: np.ndarray) -> np.ndarray:
     """The same at selected elements; ``theta_in`` holds their current stored values as doubles."""
-    acc = np.ascontiguousarray(theta_in, dtype=np.float64).copy()
-    for seed, c in zip(seeds, coeffs):
-        acc += float(c) * z_elements(t, seed, tensor_id, bits, a, b, idx)
-    return round_to(acc, t.dtype)
+    U, q, sc, ze = t._args()
+    n, sd, cf = _terms(seeds, coeffs)
+    idx = np.ascontiguousarray(idx, dtype=np.int64)
+    th = np.ascontiguousarray(theta_in, dtype=np.float64)
+    out = np.zeros(idx.size, dtype=np.float64)
+    lib().zgro_sweep_multi_elements(_p(th), ctypes.c_int(t.dtype), ctypes.c_int(n), _p(sd), _p(cf), ctypes.c_uint32(tensor_id), ctypes.c_int(bits),
+                                    _i64(t.rows), _i64(t.cols), _p(U), _i64(t.rank), _p(q), _p(sc), _p(ze), _i64(t.qrows), ctypes.c_double(a), ctypes.c_double(b),
+                                    _i64(idx.size), _p(idx), _p(out))
+    return out
+
+
+def update_coefficient(net: float, loss_plus: float, loss_minus: float, eps: float, lr: float) -> float:
+    """Coefficient of the fused restore + update sweep: -net - lr (L+ - L-)/(2 eps)  (Eq. (grad), Algorithm 1 "Update")."""
+    return float(lib().zgro_update_coefficient(ctypes.c_double(net), ctypes.c_double(loss_plus), ctypes.c_double(loss_minus),
+                                               ctypes.c_double(eps), ctypes.c_double(lr)))
+
+
+def adapt_alpha(stats: np.ndarray, a0: float, b0: float, d: int, K: int, alpha_old: float, alpha_min: float = 0.05, alpha_max: float = 0.95,
+                eta: float = 1.0) -> float:
+    """The energy-balancing candidate for the adaptive mixing ratio announced in Sec. 1 (see zgro_adapt_alpha)."""
+    st = np.ascontiguousarray(stats, dtype=np.float64).reshape(-1, 3)
+    return float(lib().zgro_adapt_alpha(_p(st), _i64(st.shape[0]), ctypes.c_double(a0), ctypes.c_double(b0), _i64(d), _i64(K),
+                                        ctypes.c_double(alpha_old), ctypes.c_double(alpha_min), ctypes.c_double(alpha_max), ctypes.c_double(eta)))
+
+
+def householder_qr(A: np.ndarray, with_r: bool = False):
+    """Orthonormal basis of the span of the columns of A (rows x r; Algorithm 1 "build basis V_r"): thin Q of a
+    Householder QR in double with R_kk > 0."""
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    rows, r = A.shape
+    Q = np.zeros((rows, r), dtype=np.float64)
+    R = np.zeros((r, r), dtype=np.float64) if with_r else None
+    lib().zgro_householder_qr(_p(A), _i64(rows), _i64(r), _p(Q), _p(R))
+    return (Q, R) if with_r else Q
 
 
 def stats_tensor(t: OracleTensor, seed: int, tensor_id: int, bits: int, a: float, b: float) -> np.ndarray:
     U, q, sc, ze = t._args()
     out = np.zeros(3, dtype=np.float64)
     lib().zgro_stats_tensor(_u64(seed), ctypes.c_uint32(tensor_id), ctypes.c_int(bits), _i64(t.rows), _i64(t.cols), _p(U), _i64(t.rank),
-                            _p(q), _p(sc), _p(ze), ctypes.c_double(a), ctypes.c_double(b), _p(out))
+                            _p(q), _p(sc), _p(ze), _i64(t.qrows), ctypes.c_double(a), ctypes.c_double(b), _p(out))
     return out
 
 
@@ -253,10 +301,16 @@ def dtc_dequantise(q: np.ndarray, scale: np.ndarray, zero: Optional[np.ndarray] 
 
 def dtc_quantise_int4(G: np.ndarray):
     """The paper's INT4 form of Sec. 3.4: unsigned codes x_q in [0, 15], lambda = (max - min)/15 and a zero
-    point delta per row, x = lambda (x_q - delta).  It is the affine quantiser above with codes and zero
-    point shifted by 8 from the signed range to the unsigned one (the dequantised values are the same)."""
-    q, sc, ze = dtc_quantise(G, bits=4, symmetric=False)
-    return (q.astype(np.int16) + 8).astype(np.int8), sc, (ze + np.float32(8.0)).astype(np.float32)
+    point delta per row, x = lambda (x_q - delta)  (zgro_dtc_quantise_row_int4)."""
+    G = np.ascontiguousarray(G, dtype=np.float64)
+    r, n = G.shape
+    q = np.zeros((r, n), dtype=np.int8)
+    sc = np.zeros(r, dtype=np.float32)
+    ze = np.zeros(r, dtype=np.float32)
+    for k in range(r):
+        lib().zgro_dtc_quantise_row_int4(_p(G[k]), _i64(n), ctypes.c_void_p(q[k].ctypes.data), ctypes.c_void_p(sc[k:].ctypes.data),
+                                         ctypes.c_void_p(ze[k:].ctypes.data))
+    return q, sc, ze
 
 
 def dtc_pack4(codes: np.ndarray) -> np.ndarray:
@@ -264,18 +318,18 @@ def dtc_pack4(codes: np.ndarray) -> np.ndarray:
     of byte j and column 2j + 1 in its high nibble (a missing last column is stored as 0)."""
     codes = np.asarray(codes)
     assert codes.ndim == 2 and codes.min() >= 0 and codes.max() <= 15
-    r, n = codes.shape
-    padded = np.zeros((r, 2 * ((n + 1) // 2)), dtype=np.uint8)
-    padded[:, :n] = codes
-    return (padded[:, 0::2] | (padded[:, 1::2] << 4)).astype(np.uint8)
+    c8 = np.ascontiguousarray(codes, dtype=np.int8)
+    r, n = c8.shape
+    out = np.zeros((r, (n + 1) // 2), dtype=np.uint8)
+    lib().zgro_dtc_pack4(_p(c8), _i64(r), _i64(n), _p(out))
+    return out
 
 
 def dtc_unpack4(packed: np.ndarray, cols: int) -> np.ndarray:
-    packed = np.asarray(packed, dtype=np.uint8)
-    out = np.zeros((packed.shape[0], 2 * packed.shape[1]), dtype=np.int8)
-    out[:, 0::2] = packed & 15
-    out[:, 1::2] = packed >> 4
-    return out[:, :cols]
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    out = np.zeros((packed.shape[0], cols), dtype=np.int8)
+    lib().zgro_dtc_unpack4(_p(packed), _i64(packed.shape[0]), _i64(cols), _p(out))
+    return out
 
 
 # ----------------------------------------------------------------------------- the call sequence
@@ -307,8 +361,7 @@ class OracleZGR:
         self.net += c
 
     def update_coefficient(self, loss_plus: float, loss_minus: float, lr: float) -> float:
-        g = projected_grad(loss_plus, loss_minus, self.eps)
-        return -self.net - lr * g
+        return update_coefficient(self.net, loss_plus, loss_minus, self.eps, lr)
 
     def sweep_multi(self, seeds: Sequence[int], coeffs: Sequence[float]) -> None:
         """One pass applying several seeds; the ledger ``self.nets`` records what stays applied per seed."""
@@ -321,7 +374,7 @@ class OracleZGR:
 
     def restore_update_multi(self, seeds: Sequence[int], loss_plus: Sequence[float], loss_minus: Sequence[float], lr: float):
         """Eq. (grad) per seed, then theta <- rnd(theta + sum_i (-net_i - lr g_i) z_i) in one pass."""
-        coeffs = [-self.nets.get(s, 0.0) - lr * projected_grad(lp, lm, self.eps) for s, lp, lm in zip(seeds, loss_plus, loss_minus)]
+        coeffs = [update_coefficient(self.nets.get(s, 0.0), lp, lm, self.eps, lr) for s, lp, lm in zip(seeds, loss_plus, loss_minus)]
         for l, t in enumerate(self.tensors):
             sweep_multi_tensor(t, seeds, coeffs, l, self.bits, self.a, self.b)
         for s in seeds:

@@ -21,7 +21,10 @@
 // Parity pins (tests/test_oracle_*.py): Philox against two independent library implementations,
 // moments/KS of the normal stream, brute-force dense construction of Eq. (perturbation),
 // span and covariance properties, exactness of the central difference on a quadratic, restore at
-// lr = 0 with double storage, DTC error bound, rounding against brute-force nearest search.
+// lr = 0 with double storage, DTC error bound, rounding against brute-force nearest search;
+// multi-seed sweeps against single sweeps, linearity and a dense construction; the Householder basis
+// against a library QR, its defining properties and a hand-worked 3 x 2 case; the adaptive mixing ratio
+// against the balance it is defined by, recomputed from the norms after the change.
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -199,13 +202,16 @@ void store_elem(void* base, int dtype, int64_t i, double v) {
 
 // Coefficient G_l[k,c]  [z_g ~ N(0, I_m), Algorithm 1 "Sample z_g"]: either the tag-1 normal at
 // element k*cols + c, or the DTC-dequantised value lambda_k (q[k,c] - delta_k)  [Sec. 3.4].
+// A proportion of the payload may arrive compressed (Sec. 3.4, the adaptive proportion omega): here the first
+// qrows rows of G_l come from the codes and the remaining rows are drawn from the seed.
 struct CoeffSource {
-  const int8_t* q;      // rank x cols, or null -> seed-generated
-  const float* scale;   // rank
-  const float* zero;    // rank or null (delta = 0)
+  const int8_t* q;      // qrows x cols, or null -> seed-generated
+  const float* scale;   // qrows
+  const float* zero;    // qrows or null (delta = 0)
+  int64_t qrows;        // rows of G_l taken from the codes (= rank when everything arrives compressed)
 };
 double coeff_at(const CoeffSource& cs, uint64_t seed, uint32_t tensor, int bits, int64_t cols, int64_t k, int64_t c) {
-  if (cs.q) {
+  if (cs.q && k < cs.qrows) {
     const double lambda = static_cast<double>(cs.scale[k]);
     const double delta = cs.zero ? static_cast<double>(cs.zero[k]) : 0.0;
     return lambda * (static_cast<double>(cs.q[k * cols + c]) - delta);
@@ -265,8 +271,8 @@ void zgro_encode(const double* src, int dtype, int64_t n, void* out) {
 // --- coefficients and perturbation ------------------------------------------------------------
 // G_l (rank x cols) as doubles.
 void zgro_coeffs(uint64_t seed, uint32_t tensor, int bits, int64_t rank, int64_t cols, const int8_t* q, const float* scale,
-                 const float* zero, double* out) {
-  const CoeffSource cs{q, scale, zero};
+                 const float* zero, int64_t qrows, double* out) {
+  const CoeffSource cs{q, scale, zero, qrows};
 #pragma omp parallel for schedule(static)
   for (int64_t k = 0; k < rank; ++k)
     for (int64_t c = 0; c < cols; ++c) out[k * cols + c] = coeff_at(cs, seed, tensor, bits, cols, k, c);
@@ -277,13 +283,13 @@ void zgro_coeffs(uint64_t seed, uint32_t tensor, int bits, int64_t rank, int64_t
 // U is rows x rank row-major (fp32 values); rank == 0 or U == null -> isotropic part only.
 // Any of z_out / iso_out / guided_out may be null.  iso_out receives a*z_iso, guided_out b*U G.
 void zgro_z_tensor(uint64_t seed, uint32_t tensor, int bits, int64_t rows, int64_t cols, const float* U, int64_t rank,
-                   const int8_t* q, const float* scale, const float* zero, double a, double b, double* z_out,
+                   const int8_t* q, const float* scale, const float* zero, int64_t qrows, double a, double b, double* z_out,
                    double* iso_out, double* guided_out) {
   const bool guided = (U != nullptr && rank > 0);
   std::vector<double> G;
   if (guided) {
     G.resize(static_cast<size_t>(rank * cols));
-    zgro_coeffs(seed, tensor, bits, rank, cols, q, scale, zero, G.data());
+    zgro_coeffs(seed, tensor, bits, rank, cols, q, scale, zero, qrows, G.data());
   }
 #pragma omp parallel for schedule(static)
   for (int64_t i = 0; i < rows; ++i) {
@@ -303,11 +309,11 @@ void zgro_z_tensor(uint64_t seed, uint32_t tensor, int bits, int64_t rows, int64
 
 // The same perturbation at selected elements (random access): idx are linear indices i*cols + c.
 void zgro_z_elements(uint64_t seed, uint32_t tensor, int bits, int64_t rows, int64_t cols, const float* U, int64_t rank,
-                     const int8_t* q, const float* scale, const float* zero, double a, double b, int64_t n_idx,
+                     const int8_t* q, const float* scale, const float* zero, int64_t qrows, double a, double b, int64_t n_idx,
                      const int64_t* idx, double* z_out) {
   (void)rows;
   const bool guided = (U != nullptr && rank > 0);
-  const CoeffSource cs{q, scale, zero};
+  const CoeffSource cs{q, scale, zero, qrows};
 #pragma omp parallel for schedule(static)
   for (int64_t t = 0; t < n_idx; ++t) {
     const int64_t e = idx[t];
@@ -328,13 +334,13 @@ void zgro_z_elements(uint64_t seed, uint32_t tensor, int bits, int64_t rows, int
 //   restore+update:  c = -net - lr * g                    [Eq. (grad); Algorithm 1 "Update"]
 // One rounding to the storage type per sweep.
 void zgro_sweep_tensor(void* theta, int dtype, uint64_t seed, uint32_t tensor, int bits, int64_t rows, int64_t cols,
-                       const float* U, int64_t rank, const int8_t* q, const float* scale, const float* zero, double a,
+                       const float* U, int64_t rank, const int8_t* q, const float* scale, const float* zero, int64_t qrows, double a,
                        double b, double c) {
   const bool guided = (U != nullptr && rank > 0);
   std::vector<double> G;
   if (guided) {
     G.resize(static_cast<size_t>(rank * cols));
-    zgro_coeffs(seed, tensor, bits, rank, cols, q, scale, zero, G.data());
+    zgro_coeffs(seed, tensor, bits, rank, cols, q, scale, zero, qrows, G.data());
   }
 #pragma omp parallel for schedule(static)
   for (int64_t i = 0; i < rows; ++i) {
@@ -356,19 +362,19 @@ void zgro_sweep_tensor(void* theta, int dtype, uint64_t seed, uint32_t tensor, i
 // (already exact in the storage type); theta_out[t] receives the rounded result.
 void zgro_sweep_elements(const double* theta_in, int dtype, uint64_t seed, uint32_t tensor, int bits, int64_t rows,
                          int64_t cols, const float* U, int64_t rank, const int8_t* q, const float* scale,
-                         const float* zero, double a, double b, double c, int64_t n_idx, const int64_t* idx,
+                         const float* zero, int64_t qrows, double a, double b, double c, int64_t n_idx, const int64_t* idx,
                          double* theta_out) {
   std::vector<double> z(static_cast<size_t>(n_idx));
-  zgro_z_elements(seed, tensor, bits, rows, cols, U, rank, q, scale, zero, a, b, n_idx, idx, z.data());
+  zgro_z_elements(seed, tensor, bits, rows, cols, U, rank, q, scale, zero, qrows, a, b, n_idx, idx, z.data());
   for (int64_t t = 0; t < n_idx; ++t) theta_out[t] = round_to(theta_in[t] + c * z[static_cast<size_t>(t)], dtype);
 }
 
 // Per-tensor energies of the two parts and of their sum: out = { sum (a z_iso)^2, sum (b U G)^2, sum z^2 }.
 void zgro_stats_tensor(uint64_t seed, uint32_t tensor, int bits, int64_t rows, int64_t cols, const float* U, int64_t rank,
-                       const int8_t* q, const float* scale, const float* zero, double a, double b, double* out3) {
+                       const int8_t* q, const float* scale, const float* zero, int64_t qrows, double a, double b, double* out3) {
   const int64_t n = rows * cols;
   std::vector<double> iso(static_cast<size_t>(n)), gd(static_cast<size_t>(n));
-  zgro_z_tensor(seed, tensor, bits, rows, cols, U, rank, q, scale, zero, a, b, nullptr, iso.data(), gd.data());
+  zgro_z_tensor(seed, tensor, bits, rows, cols, U, rank, q, scale, zero, qrows, a, b, nullptr, iso.data(), gd.data());
   double s0 = 0, s1 = 0, s2 = 0;
   for (int64_t i = 0; i < n; ++i) {
     const double x = iso[static_cast<size_t>(i)], y = gd[static_cast<size_t>(i)];
@@ -377,6 +383,136 @@ void zgro_stats_tensor(uint64_t seed, uint32_t tensor, int bits, int64_t rows, i
     s2 += (x + y) * (x + y);
   }
   out3[0] = s0; out3[1] = s1; out3[2] = s2;
+}
+
+// --- several seeds in one sweep -----------------------------------------------------------------
+// theta <- rnd_dtype(theta + sum_q c_q z(seed_q)), in place  [Algorithm 1: "Recover gradient" sums g_t z_t over
+// the seeds (and, on the edge server, over the clients), "Update" applies the sum].  One rounding to the
+// storage type for the whole sum; the terms are added in the order given.
+void zgro_sweep_multi_tensor(void* theta, int dtype, int n_terms, const uint64_t* seeds, const double* coeffs, uint32_t tensor, int bits,
+                             int64_t rows, int64_t cols, const float* U, int64_t rank, const int8_t* q, const float* scale, const float* zero,
+                             int64_t qrows, double a, double b) {
+  const bool guided = (U != nullptr && rank > 0);
+  std::vector<std::vector<double>> G(static_cast<size_t>(n_terms));
+  if (guided)
+    for (int t = 0; t < n_terms; ++t) {
+      G[static_cast<size_t>(t)].resize(static_cast<size_t>(rank * cols));
+      zgro_coeffs(seeds[t], tensor, bits, rank, cols, q, scale, zero, qrows, G[static_cast<size_t>(t)].data());
+    }
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < rows; ++i) {
+    for (int64_t col = 0; col < cols; ++col) {
+      const int64_t e = i * cols + col;
+      double acc = load_elem(theta, dtype, e);
+      for (int t = 0; t < n_terms; ++t) {
+        const double iso = a * normal_at(seeds[t], tensor, 0u, bits, static_cast<uint64_t>(e));
+        double p = 0.0;
+        if (guided)
+          for (int64_t k = 0; k < rank; ++k)
+            p += static_cast<double>(U[i * rank + k]) * G[static_cast<size_t>(t)][static_cast<size_t>(k * cols + col)];
+        const double z = iso + b * p;
+        acc += coeffs[t] * z;
+      }
+      store_elem(theta, dtype, e, round_to(acc, dtype));
+    }
+  }
+}
+
+// The same at selected elements (theta_in: their current stored values; theta_out: the rounded results).
+void zgro_sweep_multi_elements(const double* theta_in, int dtype, int n_terms, const uint64_t* seeds, const double* coeffs, uint32_t tensor,
+                               int bits, int64_t rows, int64_t cols, const float* U, int64_t rank, const int8_t* q, const float* scale,
+                               const float* zero, int64_t qrows, double a, double b, int64_t n_idx, const int64_t* idx, double* theta_out) {
+  std::vector<double> acc(theta_in, theta_in + n_idx), z(static_cast<size_t>(n_idx));
+  for (int t = 0; t < n_terms; ++t) {
+    zgro_z_elements(seeds[t], tensor, bits, rows, cols, U, rank, q, scale, zero, qrows, a, b, n_idx, idx, z.data());
+    for (int64_t j = 0; j < n_idx; ++j) acc[static_cast<size_t>(j)] += coeffs[t] * z[static_cast<size_t>(j)];
+  }
+  for (int64_t j = 0; j < n_idx; ++j) theta_out[j] = round_to(acc[static_cast<size_t>(j)], dtype);
+}
+
+// Coefficient of the fused restore + update sweep  [Eq. (grad); Algorithm 1 "Update": W <- W - eta g z]:
+// the perturbation still applied under the seed (net) is taken back and the projected-gradient step added.
+double zgro_update_coefficient(double net, double loss_plus, double loss_minus, double eps, double lr) {
+  const double g = zgro_projected_grad(loss_plus, loss_minus, eps);
+  return -net - lr * g;
+}
+
+// --- adaptive mixing ratio ------------------------------------------------------------------------
+// Sec. 1 announces that the ZGR parameter follows the relative sizes of the guided (back-propagation
+// based) and the isotropic (zeroth-order) part of the perturbation, and gives no rule.  The candidate
+// taken: balance their energies.  With the per-tensor norms  S_iso = sum (a0 Z)^2,  S_g = sum (b0 U G)^2
+// measured under the current scalars (a0, b0), the energies per unit of mixing weight are
+//   rho_iso = (S_iso / a0^2) / d    and    rho_g = (S_g / b0^2) / K        (d, K as in zgro_mix_scalars),
+// and Eq. (perturbation) with ratio alpha gives the parts the energies  alpha * s * rho_iso  and
+// (1 - alpha) * s * rho_g  (s = 1 or d by scale mode).  They are equal at
+//   alpha* = rho_g / (rho_iso + rho_g).
+// The result is damped towards the old value and clamped:  alpha = clamp((1 - eta) alpha_old + eta alpha*).
+// A part that is absent (a0 = 0, b0 = 0 or K = 0) leaves alpha unchanged.
+double zgro_adapt_alpha(const double* stats3, int64_t n_tensors, double a0, double b0, int64_t d, int64_t K, double alpha_old,
+                        double alpha_min, double alpha_max, double eta) {
+  if (a0 == 0.0 || b0 == 0.0 || K <= 0) return alpha_old;
+  double s_iso = 0.0, s_g = 0.0;
+  for (int64_t l = 0; l < n_tensors; ++l) {
+    s_iso += stats3[3 * l + 0];
+    s_g += stats3[3 * l + 1];
+  }
+  const double rho_iso = s_iso / (a0 * a0) / static_cast<double>(d);
+  const double rho_g = s_g / (b0 * b0) / static_cast<double>(K);
+  if (!(rho_iso + rho_g > 0.0)) return alpha_old;
+  const double target = rho_g / (rho_iso + rho_g);
+  const double mixed = (1.0 - eta) * alpha_old + eta * target;
+  return std::fmin(std::fmax(mixed, alpha_min), alpha_max);
+}
+
+// --- subspace construction ------------------------------------------------------------------------
+// Algorithm 1 "Collect gradients to build basis V_r" (Sec. 3.2): an orthonormal basis of the span of the
+// last r gradients of a tensor.  A is rows x r (column j = gradient j, row-major storage); Householder QR in
+// double, A = Q R with R upper triangular; the thin Q (rows x r) is returned with the sign convention
+// R_kk > 0, which makes it unique for a full-rank A.  R (r x r, row-major) is returned if R_out is not null.
+void zgro_householder_qr(const double* A, int64_t rows, int64_t r, double* Q_out, double* R_out) {
+  std::vector<double> W(A, A + rows * r);                       // working copy, becomes R in its upper triangle
+  std::vector<double> V(static_cast<size_t>(rows * r), 0.0);    // Householder vectors, column k in V[:, k]
+  std::vector<double> beta(static_cast<size_t>(r), 0.0);
+  for (int64_t k = 0; k < r; ++k) {
+    double norm2 = 0.0;
+    for (int64_t i = k; i < rows; ++i) norm2 += W[static_cast<size_t>(i * r + k)] * W[static_cast<size_t>(i * r + k)];
+    const double norm = std::sqrt(norm2);
+    if (norm == 0.0) continue;
+    const double x0 = W[static_cast<size_t>(k * r + k)];
+    const double alpha = x0 >= 0.0 ? -norm : norm;            // reflect x onto alpha e_k, away from x0 (no cancellation)
+    double vnorm2 = 0.0;
+    for (int64_t i = k; i < rows; ++i) {
+      double v = W[static_cast<size_t>(i * r + k)];
+      if (i == k) v -= alpha;
+      V[static_cast<size_t>(i * r + k)] = v;
+      vnorm2 += v * v;
+    }
+    beta[static_cast<size_t>(k)] = vnorm2 > 0.0 ? 2.0 / vnorm2 : 0.0;
+    for (int64_t j = k; j < r; ++j) {                          // W <- (I - beta v v^T) W on the trailing columns
+      double dot = 0.0;
+      for (int64_t i = k; i < rows; ++i) dot += V[static_cast<size_t>(i * r + k)] * W[static_cast<size_t>(i * r + j)];
+      const double f = beta[static_cast<size_t>(k)] * dot;
+      for (int64_t i = k; i < rows; ++i) W[static_cast<size_t>(i * r + j)] -= f * V[static_cast<size_t>(i * r + k)];
+    }
+  }
+  // Q = H_0 H_1 ... H_{r-1} applied to the first r columns of the identity
+  std::vector<double> Q(static_cast<size_t>(rows * r), 0.0);
+  for (int64_t j = 0; j < r && j < rows; ++j) Q[static_cast<size_t>(j * r + j)] = 1.0;
+  for (int64_t k = r - 1; k >= 0; --k) {
+    for (int64_t j = 0; j < r; ++j) {
+      double dot = 0.0;
+      for (int64_t i = k; i < rows; ++i) dot += V[static_cast<size_t>(i * r + k)] * Q[static_cast<size_t>(i * r + j)];
+      const double f = beta[static_cast<size_t>(k)] * dot;
+      for (int64_t i = k; i < rows; ++i) Q[static_cast<size_t>(i * r + j)] -= f * V[static_cast<size_t>(i * r + k)];
+    }
+  }
+  // sign convention: R_kk > 0
+  for (int64_t k = 0; k < r; ++k) {
+    const double sgn = W[static_cast<size_t>(k * r + k)] < 0.0 ? -1.0 : 1.0;
+    for (int64_t i = 0; i < rows; ++i) Q_out[i * r + k] = sgn * Q[static_cast<size_t>(i * r + k)];
+    if (R_out)
+      for (int64_t j = 0; j < r; ++j) R_out[k * r + j] = j >= k ? sgn * W[static_cast<size_t>(k * r + j)] : 0.0;
+  }
 }
 
 // --- DTC (Sec. 3.4) ---------------------------------------------------------------------------
@@ -414,6 +550,35 @@ void zgro_dtc_quantise_row(const double* x, int64_t n, int bits, int symmetric, 
 
 void zgro_dtc_dequantise_row(const int8_t* q, int64_t n, float scale, float zero, double* out) {
   for (int64_t i = 0; i < n; ++i) out[i] = static_cast<double>(scale) * (static_cast<double>(q[i]) - static_cast<double>(zero));
+}
+
+// The paper's INT4 payload of Sec. 3.4: unsigned codes x_q in [0, 15], lambda = (max - min)/15 and a zero point
+// per row, x = lambda (x_q - delta).  It is the affine 4-bit quantiser above with codes and zero point moved by
+// 8 from the signed range [-8, 7] to the unsigned one (the dequantised values are unchanged).
+void zgro_dtc_quantise_row_int4(const double* x, int64_t n, int8_t* q_out, float* scale_out, float* zero_out) {
+  zgro_dtc_quantise_row(x, n, 4, 0, q_out, scale_out, zero_out);
+  for (int64_t i = 0; i < n; ++i) q_out[i] = static_cast<int8_t>(q_out[i] + 8);
+  *zero_out = *zero_out + 8.0f;
+}
+
+// Transmission layout of 4-bit codes: a row of `cols` codes becomes (cols + 1)/2 bytes, column 2j in the low
+// nibble of byte j and column 2j + 1 in its high nibble; a missing last column is stored as 0.
+void zgro_dtc_pack4(const int8_t* codes, int64_t rows, int64_t cols, uint8_t* out) {
+  const int64_t nb = (cols + 1) / 2;
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t j = 0; j < nb; ++j) {
+      const unsigned lo = static_cast<unsigned>(codes[r * cols + 2 * j]) & 15u;
+      const unsigned hi = (2 * j + 1 < cols) ? (static_cast<unsigned>(codes[r * cols + 2 * j + 1]) & 15u) : 0u;
+      out[r * nb + j] = static_cast<uint8_t>(lo | (hi << 4));
+    }
+}
+void zgro_dtc_unpack4(const uint8_t* packed, int64_t rows, int64_t cols, int8_t* out) {
+  const int64_t nb = (cols + 1) / 2;
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t c = 0; c < cols; ++c) {
+      const unsigned byte = packed[r * nb + c / 2];
+      out[r * cols + c] = static_cast<int8_t>((c & 1) ? (byte >> 4) : (byte & 15u));
+    }
 }
 
 int zgro_num_threads(void) {

@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libzgr.so")
-SOURCES = ["zgr_host.cu", "zgr_kernels.cu", "zgr_noalloc.cu", "zgr_umma.cu"]
+SOURCES = ["zgr_host.cu", "zgr_kernels.cu", "zgr_noalloc.cu", "zgr_subspace.cu", "zgr_umma.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -272,7 +272,7 @@ struct Storage<__nv_bfloat16> {
 template <int BITS, bool PRECISE>
 __device__ __forceinline__ void coeffs8(const TensorDesc& td, const PhiloxKeys& keys, const NormalScale& unit, float cb, int k,
                                         int64_t c, float (&g)[8]) {
-  if (td.q != nullptr) {
+  if (td.q != nullptr && k < td.qrows) {
     const float lambda = td.qscale[k] * cb;
     const float delta = td.qzero ? td.qzero[k] : 0.0f;
     if (td.qbits == 4) {
@@ -299,7 +299,7 @@ __device__ __forceinline__ void coeffs8(const TensorDesc& td, const PhiloxKeys& 
 
 template <int BITS, bool PRECISE>
 __device__ __forceinline__ float coeff1(const TensorDesc& td, const PhiloxKeys& keys, const NormalScale& unit, float cb, int k, int64_t c) {
-  if (td.q != nullptr) {
+  if (td.q != nullptr && k < td.qrows) {
     const float delta = td.qzero ? td.qzero[k] : 0.0f;
     float code;
     if (td.qbits == 4) {
@@ -345,13 +345,13 @@ __device__ __forceinline__ float iso1(const SweepParams& p, uint32_t tensor, uin
   return z;
 }
 
-// sum_q c_q b G_q[k][c .. c+7].  Compressed coefficients do not depend on the seed: they are scaled
-// by the sum of the terms' factors.
+// sum_q c_q b G_q[k][c .. c+7].  Compressed coefficients (rows below td.qrows) do not depend on the seed: they
+// are scaled by the sum of the terms' factors.
 template <int BITS, bool PRECISE, bool MULTI>
 __device__ __forceinline__ void guided8(const TensorDesc& td, const SweepParams& p, int k, int64_t c, float (&g)[8]) {
   if (!MULTI) {
     coeffs8<BITS, PRECISE>(td, p.term[0].keys, p.unit, p.term[0].cb, k, c, g);
-  } else if (td.q != nullptr) {
+  } else if (td.q != nullptr && k < td.qrows) {
     float cb = 0.0f;
     for (int q = 0; q < p.n_terms; ++q) cb += p.term[q].cb;
     coeffs8<BITS, PRECISE>(td, p.term[0].keys, p.unit, cb, k, c, g);
@@ -370,7 +370,7 @@ __device__ __forceinline__ void guided8(const TensorDesc& td, const SweepParams&
 template <int BITS, bool PRECISE, bool MULTI>
 __device__ __forceinline__ float guided1(const TensorDesc& td, const SweepParams& p, int k, int64_t c) {
   if (!MULTI) return coeff1<BITS, PRECISE>(td, p.term[0].keys, p.unit, p.term[0].cb, k, c);
-  if (td.q != nullptr) {
+  if (td.q != nullptr && k < td.qrows) {
     float cb = 0.0f;
     for (int q = 0; q < p.n_terms; ++q) cb += p.term[q].cb;
     return coeff1<BITS, PRECISE>(td, p.term[0].keys, p.unit, cb, k, c);

@@ -15,6 +15,7 @@
 #include "zgr_internal.h"
 #include "zgr_host_internal.h"
 #include "zgr_kernels.h"
+#include "zgr_subspace.h"
 
 using namespace zgr;
 
@@ -26,6 +27,7 @@ struct Group {
   WorkItem* d_items = nullptr;
   int grid = 0;
   int64_t elements = 0;                                   // weights covered by one launch
+  std::vector<int32_t> first_item;                        // per tensor l: index of its first item in `items` (size n + 1; items are in tensor order)
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed;  // per-launch events while profiling is on
 };
 
@@ -62,6 +64,9 @@ struct zgr_ctx {
   CUtensorMap* d_tmaps = nullptr;     // three per tensor (theta, U hi, U lo); tcgen05 path only
   std::vector<CUtensorMap> tmaps;     // host mirror
   int* d_err = nullptr;               // set by a kernel whose bounded wait gave up
+  std::vector<cudaEvent_t> layer_events;  // zgr_perturb_layers: one per layer plus one, created on first use
+  void* d_qr = nullptr;               // scratch of zgr_build_subspace (grown on demand)
+  size_t qr_bytes = 0;
 };
 
 namespace {
@@ -88,6 +93,14 @@ NormalScale make_scale(double s, int bits) {
   ns.phase = static_cast<float>(kTwoPi * off + (s >= 0 ? -kTwoPi : -0.5 * kTwoPi));
   ns.u1_off = static_cast<float>(off);
   return ns;
+}
+
+// Power of two that brings the coefficient strips of the tcgen05 kernel near 1: the smallest k with
+// cb 2^k >= 1/2, cb = sum_q |c_q| b (0 if there is no guided part in this call).
+int kshift_for(double cb) {
+  if (!(cb > 0.0) || !std::isfinite(cb)) return 0;
+  const int k = static_cast<int>(std::ceil(-std::log2(cb))) - 1;
+  return std::min(std::max(k, -24), 40);
 }
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -209,6 +222,14 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
     for (const WorkItem& w : g.items) g.elements += g.kc.path == PATH_ISO ? w.nrows_or_count : w.nrows_or_count * w.ncols;
   }
   for (Group& g : out) g.grid = static_cast<int>(std::min<int64_t>(static_cast<int64_t>(g.items.size()), static_cast<int64_t>(sm_count) * blocks_per_sm(g.kc.path)));
+  // tensors were visited in ascending order, so each tensor's items are contiguous within its group
+  for (Group& g : out) {
+    g.first_item.assign(descs.size() + 1, static_cast<int32_t>(g.items.size()));
+    for (size_t i = g.items.size(); i-- > 0;) g.first_item[static_cast<size_t>(g.items[i].tensor)] = static_cast<int32_t>(i);
+    for (size_t l = descs.size(); l-- > 0;)
+      if (g.first_item[l] > g.first_item[l + 1]) g.first_item[l] = g.first_item[l + 1];   // tensors without items in this group
+    // (after the two passes first_item is non-decreasing and [first_item[l], first_item[l+1]) are the items of tensor l)
+  }
 }
 
 int check(zgr_ctx* ctx, cudaError_t e) {
@@ -240,7 +261,9 @@ int upload_groups(zgr_ctx* ctx, std::vector<Group>& groups) {
 }
 
 // One sweep  theta <- rnd(theta + sum_q c_q z(seed_q))  over the planned groups (n terms, 1 <= n <= kMaxTerms).
-int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, int n, const uint64_t* seeds, const double* c, cudaStream_t st) {
+// t0 <= t1 restricts the sweep to the tensors [t0, t1) (layer-wise sweeps); t1 < 0 means all of them.
+int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, int n, const uint64_t* seeds, const double* c, cudaStream_t st,
+          int32_t t0 = 0, int32_t t1 = -1) {
   SweepParams p;
   std::memset(&p, 0, sizeof(p));
   for (int q = 0; q < n; ++q) {
@@ -252,19 +275,37 @@ int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, i
   p.unit = make_scale(1.0, ctx->cfg.bits_per_normal);
   p.tensors = d_descs;
   p.stats = nullptr;
+  double cb_total = 0.0;
+  for (int q = 0; q < n; ++q) cb_total += std::fabs(c[q] * ctx->b);
+  p.kshift = kshift_for(cb_total);
   for (Group& g : groups) {
     if (g.items.empty()) continue;
     p.items = g.d_items;
     p.n_items = static_cast<int32_t>(g.items.size());
+    int grid = g.grid;
+    if (t1 >= 0) {
+      const int32_t b0 = g.first_item[static_cast<size_t>(t0)], b1 = g.first_item[static_cast<size_t>(t1)];
+      if (b1 <= b0) continue;
+      p.items = g.d_items + b0;
+      p.n_items = b1 - b0;
+      grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * blocks_per_sm(g.kc.path)));
+    }
     cudaEvent_t e0 = nullptr, e1 = nullptr;
-    if (ctx->profiling) {
-      if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return check(ctx, cudaErrorUnknown);
+    if (ctx->profiling && t1 < 0) {
+      if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        return check(ctx, cudaErrorUnknown);
+      }
       cudaEventRecord(e0, st);
     }
-    const int rc = check(ctx, g.kc.path == PATH_UMMA ? launch_sweep_umma(g.kc, p, ctx->d_tmaps, ctx->d_err, g.grid, st)
-                                                     : launch_sweep(g.kc, p, g.grid, st));
-    if (rc != ZGR_OK) return rc;
-    if (ctx->profiling) {
+    const int rc = check(ctx, g.kc.path == PATH_UMMA ? launch_sweep_umma(g.kc, p, ctx->d_tmaps, ctx->d_err, grid, st)
+                                                     : launch_sweep(g.kc, p, grid, st));
+    if (rc != ZGR_OK) {
+      if (e0) cudaEventDestroy(e0);
+      if (e1) cudaEventDestroy(e1);
+      return rc;
+    }
+    if (e0) {
       cudaEventRecord(e1, st);
       g.timed.emplace_back(e0, e1);
     }
@@ -281,6 +322,15 @@ int flush_descs(zgr_ctx* ctx, cudaStream_t st) {
 }
 
 bool is_finite(double x) { return std::isfinite(x); }
+
+// A context's tables, tensor maps and borrowed pointers live on the device that was current at zgr_init.
+// Launching from another current device would hand its kernels foreign addresses, so every entry point
+// that enqueues work checks this first and refuses before anything is launched.
+bool on_ctx_device(const zgr_ctx* ctx) {
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess) return false;
+  return zgr_debug_check_device(ctx->device, cur) == ZGR_OK;
+}
 
 // Mixing scalars of Eq. (perturbation) with n := d and m := K
 void set_mixing(zgr_ctx* ctx, double alpha) {
@@ -348,13 +398,14 @@ std::vector<Group>& multi_groups(zgr_ctx* ctx, int* rc) {
 namespace zgr {
 PhiloxKeys host_make_keys(uint64_t seed) { return make_keys(seed); }
 NormalScale host_make_scale(double s, int bits) { return make_scale(s, bits); }
-bool host_ctx_view(const zgr_ctx* ctx, int32_t l, TensorDesc* desc, double* a, double* b, int* bits, int* sticky) {
+bool host_ctx_view(const zgr_ctx* ctx, int32_t l, TensorDesc* desc, double* a, double* b, int* bits, int* sticky, int* device) {
   if (!ctx || l < 0 || l >= static_cast<int32_t>(ctx->descs.size())) return false;
   *desc = ctx->descs[static_cast<size_t>(l)];
   *a = ctx->a;
   *b = ctx->b;
   *bits = ctx->cfg.bits_per_normal;
   *sticky = ctx->sticky;
+  *device = ctx->device;
   return true;
 }
 }  // namespace zgr
@@ -399,6 +450,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
     td.qscale = nullptr;
     td.qzero = nullptr;
     td.qbits = 8;
+    td.qrows = 0;
     td.rows = t.rows;
     td.cols = t.cols;
     td.rank = t.rank;
@@ -406,6 +458,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
     td.id = l;
     td.dtype = t.dtype;
     td.umma = 0;
+    td.ushift = 0;
     td.Uhi = nullptr;
     td.Ulo = nullptr;
     const bool vec = (reinterpret_cast<uintptr_t>(t.data) & 15) == 0 && (t.cols % 8 == 0);
@@ -422,10 +475,13 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
       // tcgen05 + TMA path: row-major hi/lo copies of U and three tensor maps
       if (rc == ZGR_OK && umma_wanted() && encode_tiled_fn() != nullptr && t.rows < (int64_t{1} << 31) - 256 && t.cols < (int64_t{1} << 31) - 256) {
         const int64_t rows_pad = ((t.rows + 127) / 128) * 128;
+        // entries of an orthonormal U are about 1/sqrt(rows): scaled by 2^ushift they sit between 1 and 2 in size
+        // (capped at 2^12, which leaves fp16 room for entries up to 16 in size)
+        td.ushift = std::min<int32_t>(12, static_cast<int32_t>(std::ceil(0.5 * std::log2(static_cast<double>(t.rows)))));
         uint16_t *hi = nullptr, *lo = nullptr;
         rc = dev_alloc(ctx, &hi, static_cast<size_t>(rows_pad) * td.kpad);
         if (rc == ZGR_OK) rc = dev_alloc(ctx, &lo, static_cast<size_t>(rows_pad) * td.kpad);
-        if (rc == ZGR_OK) rc = check(ctx, launch_split_subspace_rowmajor(t.U, t.rows, t.rank, td.kpad, rows_pad, hi, lo, nullptr));
+        if (rc == ZGR_OK) rc = check(ctx, launch_split_subspace_rowmajor(t.U, t.rows, t.rank, td.kpad, rows_pad, td.ushift, hi, lo, nullptr));
         if (rc == ZGR_OK) {
           ctx->launches++;
           CUtensorMap* m = &ctx->tmaps[static_cast<size_t>(3 * l)];
@@ -442,7 +498,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
   if (rc == ZGR_OK) {
     std::vector<SplitJob> jobs;
     for (const TensorDesc& td : ctx->descs)
-      if (td.umma) jobs.push_back(SplitJob{td.U, td.Uhi, td.Ulo, td.rows, ((td.rows + 127) / 128) * 128, td.rank, td.kpad});
+      if (td.umma) jobs.push_back(SplitJob{td.U, td.Uhi, td.Ulo, td.rows, ((td.rows + 127) / 128) * 128, td.rank, td.kpad, td.ushift});
     ctx->n_split_jobs = static_cast<int>(jobs.size());
     if (!jobs.empty()) {
       rc = dev_alloc(ctx, &ctx->d_split_jobs, jobs.size());
@@ -475,6 +531,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
 int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream) {
   if (!ctx || !is_finite(scale)) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   if (!ctx->ledger.empty() && !(ctx->ledger.size() == 1 && ctx->ledger.count(seed) == 1)) return ZGR_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = flush_descs(ctx, st);
@@ -488,6 +545,7 @@ int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream) {
 int zgr_restore_update(zgr_ctx* ctx, uint64_t seed, double loss_plus, double loss_minus, double lr, void* stream) {
   if (!ctx || !is_finite(loss_plus) || !is_finite(loss_minus) || !is_finite(lr)) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   const auto active = ctx->ledger.find(seed);
   if (active == ctx->ledger.end()) return ZGR_ESTATE;
   // Eq. (grad): projected gradient; Algorithm 1 "Update": W <- W - eta g z, fused with the restore
@@ -512,6 +570,7 @@ int zgr_sweep_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, const double
       if (seeds[j] == seeds[i]) return ZGR_EINVAL;
   }
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
@@ -538,6 +597,7 @@ int zgr_restore_update_multi(zgr_ctx* ctx, int32_t n, const uint64_t* seeds, con
     if (!is_finite(c[i])) return ZGR_EINVAL;
   }
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
@@ -561,17 +621,119 @@ int zgr_set_alpha(zgr_ctx* ctx, double alpha) {
   return ZGR_OK;
 }
 
-int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits) {
+int zgr_adapt_alpha(zgr_ctx* ctx, const double* stats, double alpha_min, double alpha_max, double eta, double* alpha_out) {
+  if (!ctx || !stats || !alpha_out) return ZGR_EINVAL;
+  if (!(alpha_min >= 0.0 && alpha_min <= alpha_max && alpha_max <= 1.0) || !(eta >= 0.0 && eta <= 1.0)) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (!ctx->ledger.empty()) return ZGR_ESTATE;
+  const double alpha_old = ctx->cfg.alpha;
+  *alpha_out = alpha_old;
+  // Energy of each part per unit of its mixing weight, from the norms measured under the current (a, b):
+  // sum (a Z)^2 / a^2 per parameter and sum (b U G)^2 / b^2 per guided coefficient.  Eq. (perturbation) gives
+  // the parts the weights alpha/d and (1 - alpha)/K (times d in the unit normalisation), so their energies
+  // are equal where alpha / (1 - alpha) = e_g / e_iso.  A part that is switched off cannot be measured:
+  // the ratio then stays as it is.
+  if (ctx->a == 0.0 || ctx->b == 0.0 || ctx->K == 0) return ZGR_OK;
+  double iso = 0.0, guided = 0.0;
+  for (size_t l = 0; l < ctx->descs.size(); ++l) {
+    if (!is_finite(stats[3 * l]) || !is_finite(stats[3 * l + 1]) || stats[3 * l] < 0.0 || stats[3 * l + 1] < 0.0) return ZGR_EINVAL;
+    iso += stats[3 * l];
+    guided += stats[3 * l + 1];
+  }
+  const double e_iso = iso / (ctx->a * ctx->a) / static_cast<double>(ctx->d);
+  const double e_g = guided / (ctx->b * ctx->b) / static_cast<double>(ctx->K);
+  if (!(e_iso + e_g > 0.0)) return ZGR_OK;
+  double alpha = (1.0 - eta) * alpha_old + eta * (e_g / (e_iso + e_g));
+  alpha = std::min(std::max(alpha, alpha_min), alpha_max);
+  set_mixing(ctx, alpha);
+  *alpha_out = alpha;
+  return ZGR_OK;
+}
+
+int zgr_set_coeffs_dtc_rows(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits, int32_t n_rows) {
   if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
   if (!q || !scale || (bits != 8 && bits != 4)) return ZGR_EINVAL;
   TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
-  if (td.rank == 0) return ZGR_EINVAL;
+  if (td.rank == 0 || n_rows < 1 || n_rows > td.rank) return ZGR_EINVAL;
   if (!ctx->ledger.empty()) return ZGR_ESTATE;
   td.q = q;
   td.qscale = scale;
   td.qzero = zero;
   td.qbits = bits;
+  td.qrows = n_rows;
   ctx->descs_dirty = true;
+  return ZGR_OK;
+}
+
+int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits) {
+  if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
+  return zgr_set_coeffs_dtc_rows(ctx, tensor, q, scale, zero, bits, ctx->descs[static_cast<size_t>(tensor)].rank);
+}
+
+int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_layers, const int32_t* layer_end, int32_t n_deliveries,
+                       const zgr_coeff_delivery* deliveries, void* stream, void* copy_stream) {
+  if (!ctx || !is_finite(scale) || n_layers < 1 || !layer_end || n_deliveries < 0 || (n_deliveries > 0 && !deliveries)) return ZGR_EINVAL;
+  const int32_t n = static_cast<int32_t>(ctx->descs.size());
+  for (int32_t L = 0; L < n_layers; ++L)
+    if (layer_end[L] <= (L ? layer_end[L - 1] : 0) || layer_end[L] > n) return ZGR_EINVAL;
+  if (layer_end[n_layers - 1] != n) return ZGR_EINVAL;
+  // which layer each delivery belongs to; every delivery must name a tensor whose compressed coefficients are set
+  std::vector<std::vector<int32_t>> by_layer(static_cast<size_t>(n_layers));
+  std::vector<char> seen(static_cast<size_t>(n), 0);
+  for (int32_t i = 0; i < n_deliveries; ++i) {
+    const zgr_coeff_delivery& d = deliveries[i];
+    if (d.tensor < 0 || d.tensor >= n || seen[static_cast<size_t>(d.tensor)] || !d.q || !d.scale) return ZGR_EINVAL;
+    seen[static_cast<size_t>(d.tensor)] = 1;
+    const TensorDesc& td = ctx->descs[static_cast<size_t>(d.tensor)];
+    if (td.q == nullptr || (d.zero != nullptr) != (td.qzero != nullptr)) return ZGR_EINVAL;
+    const int32_t L = static_cast<int32_t>(std::upper_bound(layer_end, layer_end + n_layers, d.tensor) - layer_end);
+    by_layer[static_cast<size_t>(L)].push_back(i);
+  }
+  if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
+  if (!ctx->ledger.empty() && (n_deliveries > 0 || !(ctx->ledger.size() == 1 && ctx->ledger.count(seed) == 1))) return ZGR_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream), cs = static_cast<cudaStream_t>(copy_stream);
+  int rc = flush_descs(ctx, st);
+  if (rc != ZGR_OK) return rc;
+  while (ctx->layer_events.size() < static_cast<size_t>(n_layers) + 1) {
+    cudaEvent_t e = nullptr;
+    rc = check(ctx, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    if (rc != ZGR_OK) return rc;
+    ctx->layer_events.push_back(e);
+  }
+  if (n_deliveries > 0) {
+    // The copies may not overtake work already enqueued on `stream` that still reads the destination buffers.
+    rc = check(ctx, cudaEventRecord(ctx->layer_events[static_cast<size_t>(n_layers)], st));
+    if (rc == ZGR_OK) rc = check(ctx, cudaStreamWaitEvent(cs, ctx->layer_events[static_cast<size_t>(n_layers)], 0));
+    if (rc != ZGR_OK) return rc;
+    // All copies are enqueued up front, layer by layer: the copy engine runs ahead of the sweeps as far as it can,
+    // so layer l + 1 (and later ones) travel while layer l is swept (Sec. 3.3).
+    for (int32_t L = 0; L < n_layers; ++L) {
+      if (by_layer[static_cast<size_t>(L)].empty()) continue;
+      for (int32_t i : by_layer[static_cast<size_t>(L)]) {
+        const zgr_coeff_delivery& d = deliveries[i];
+        const TensorDesc& td = ctx->descs[static_cast<size_t>(d.tensor)];
+        const size_t row_bytes = td.qbits == 4 ? static_cast<size_t>((td.cols + 1) / 2) : static_cast<size_t>(td.cols);
+        rc = check(ctx, cudaMemcpyAsync(const_cast<int8_t*>(td.q), d.q, row_bytes * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
+        if (rc == ZGR_OK)
+          rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.qscale), d.scale, sizeof(float) * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
+        if (rc == ZGR_OK && d.zero)
+          rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.qzero), d.zero, sizeof(float) * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
+        if (rc != ZGR_OK) return rc;
+      }
+      rc = check(ctx, cudaEventRecord(ctx->layer_events[static_cast<size_t>(L)], cs));
+      if (rc != ZGR_OK) return rc;
+    }
+  }
+  for (int32_t L = 0; L < n_layers; ++L) {
+    if (n_deliveries > 0 && !by_layer[static_cast<size_t>(L)].empty()) {
+      rc = check(ctx, cudaStreamWaitEvent(st, ctx->layer_events[static_cast<size_t>(L)], 0));
+      if (rc != ZGR_OK) return rc;
+    }
+    rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, st, L ? layer_end[L - 1] : 0, layer_end[L]);
+    if (rc != ZGR_OK) return rc;   // (a failure here leaves the earlier layers swept: the context is sticky-failed by check())
+  }
+  ledger_add(ctx, seed, scale);
   return ZGR_OK;
 }
 
@@ -583,6 +745,7 @@ int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor) {
   td.q = nullptr;
   td.qscale = nullptr;
   td.qzero = nullptr;
+  td.qrows = 0;
   ctx->descs_dirty = true;
   return ZGR_OK;
 }
@@ -590,6 +753,7 @@ int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor) {
 int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
   if (!ctx || !out) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
@@ -628,6 +792,7 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
   p.items = ctx->d_stats_items;
   p.n_items = static_cast<int32_t>(ctx->stats_items.size());
   p.term[0].cb = static_cast<float>(ctx->b);
+  p.kshift = kshift_for(std::fabs(ctx->b));
   p.stats = ctx->d_stats;
   if (p.n_items > 0) {
     const int grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * 4));
@@ -653,6 +818,7 @@ int zgr_debug_philox(zgr_ctx* ctx, uint64_t seed, int32_t tensor, int32_t tag, u
   if (!ctx || !dev_out || n_blocks < 0 || tensor < 0 || tag < 0) return ZGR_EINVAL;
   if (reinterpret_cast<uintptr_t>(dev_out) % 16 != 0) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   if (n_blocks == 0) return ZGR_OK;
   const int rc = check(ctx, launch_philox_blocks(make_keys(seed), static_cast<uint32_t>(tensor), static_cast<uint32_t>(tag), first_block, n_blocks,
                                                  dev_out, static_cast<cudaStream_t>(stream)));
@@ -664,6 +830,7 @@ int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, voi
   if (!ctx || !dev_out || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
   if (reinterpret_cast<uintptr_t>(dev_out) % 4 != 0) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (ctx->frag_stale[static_cast<size_t>(tensor)]) {
     const TensorDesc& cur = ctx->descs[static_cast<size_t>(tensor)];
@@ -692,11 +859,76 @@ int zgr_debug_z(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, voi
   return rc;
 }
 
+int zgr_debug_z_tcgen05(zgr_ctx* ctx, uint64_t seed, int32_t tensor, float* dev_out, void* stream) {
+  if (!ctx || !dev_out || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
+  if (reinterpret_cast<uintptr_t>(dev_out) % 16 != 0) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
+  const TensorDesc& cur = ctx->descs[static_cast<size_t>(tensor)];
+  if (!cur.umma || !ctx->guided_at_init) return ZGR_ESTATE;   // the sweeps do not serve this tensor with the tcgen05 kernel
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = flush_descs(ctx, st);
+  if (rc != ZGR_OK) return rc;
+  // A one-tensor model whose weights are a zeroed 16-bit image, swept once with coefficient 1 by the tcgen05
+  // kernel itself; its fp32 results go to dev_out instead of being rounded into the image.
+  const size_t owned_before = ctx->owned.size();
+  const size_t numel = static_cast<size_t>(cur.rows * cur.cols);
+  uint16_t* image = nullptr;
+  CUtensorMap* d_maps = nullptr;
+  TensorDesc* d_one = nullptr;
+  std::vector<Group> groups;
+  rc = dev_alloc(ctx, &image, numel);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemsetAsync(image, 0, numel * sizeof(uint16_t), st));
+  CUtensorMap maps[3];
+  if (rc == ZGR_OK) {
+    maps[1] = ctx->tmaps[static_cast<size_t>(3 * tensor + 1)];
+    maps[2] = ctx->tmaps[static_cast<size_t>(3 * tensor + 2)];
+    if (!make_map_16bit(&maps[0], image, cur.rows, cur.cols, 64)) rc = check(ctx, cudaErrorUnknown);
+  }
+  if (rc == ZGR_OK) rc = dev_alloc(ctx, &d_maps, 3);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemcpyAsync(d_maps, maps, sizeof(maps), cudaMemcpyHostToDevice, st));
+  std::vector<TensorDesc> one(1, cur);
+  one[0].data = image;
+  if (rc == ZGR_OK) rc = dev_alloc(ctx, &d_one, 1);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemcpyAsync(d_one, one.data(), sizeof(TensorDesc), cudaMemcpyHostToDevice, st));
+  if (rc == ZGR_OK) {
+    plan(one, std::vector<int>(1, 0), true, ctx->cfg.bits_per_normal, ctx->sm_count, groups);
+    rc = upload_groups(ctx, groups);
+  }
+  if (rc == ZGR_OK) {
+    SweepParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.term[0].keys = make_keys(seed);
+    p.term[0].iso = make_scale(ctx->a, ctx->cfg.bits_per_normal);
+    p.term[0].cb = static_cast<float>(ctx->b);
+    p.n_terms = 1;
+    p.unit = make_scale(1.0, ctx->cfg.bits_per_normal);
+    p.tensors = d_one;
+    p.zout = dev_out;
+    p.kshift = kshift_for(std::fabs(ctx->b));
+    for (Group& g : groups) {
+      if (g.items.empty()) continue;
+      if (g.kc.path != PATH_UMMA) { rc = ZGR_ESTATE; break; }
+      p.items = g.d_items;
+      p.n_items = static_cast<int32_t>(g.items.size());
+      rc = check(ctx, launch_debug_z_umma(g.kc, p, d_maps, ctx->d_err, g.grid, st));
+      if (rc != ZGR_OK) break;
+      ctx->launches++;
+    }
+  }
+  const int rc_sync = check(ctx, cudaStreamSynchronize(st));
+  if (rc == ZGR_OK) rc = rc_sync;
+  for (size_t i = owned_before; i < ctx->owned.size(); ++i) cudaFree(ctx->owned[i]);
+  ctx->owned.resize(owned_before);
+  return rc;
+}
+
 int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_t src_is_host, void* stream) {
   if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
   TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
   if (td.rank == 0) return ZGR_EINVAL;
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   if (!ctx->ledger.empty()) return ZGR_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = ZGR_OK;
@@ -717,10 +949,52 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
   }
   if (rc == ZGR_OK && td.umma) {
     const int64_t rows_pad = ((td.rows + 127) / 128) * 128;
-    rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.Uhi, td.Ulo, st));
+    rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.ushift, td.Uhi, td.Ulo, st));
     if (rc == ZGR_OK) ctx->launches++;
   }
   return rc;
+}
+
+int zgr_build_subspace(zgr_ctx* ctx, int32_t tensor, const float* grads, int32_t src_is_host, void* stream) {
+  if (!ctx || tensor < 0 || tensor >= static_cast<int32_t>(ctx->descs.size())) return ZGR_EINVAL;
+  TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
+  if (td.rank == 0 || td.rows < td.rank) return ZGR_EINVAL;
+  if (grads && reinterpret_cast<uintptr_t>(grads) % 4 != 0) return ZGR_EINVAL;
+  if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
+  if (!ctx->ledger.empty()) return ZGR_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t need = subspace_scratch_bytes(td.rows, td.rank);
+  if (need > ctx->qr_bytes) {
+    void* q = nullptr;
+    const int rc = check(ctx, cudaMalloc(&q, need));
+    if (rc != ZGR_OK) return rc;
+    ctx->owned.push_back(q);          // an outgrown scratch buffer stays owned until zgr_destroy; work enqueued on it may still run
+    ctx->d_qr = q;
+    ctx->qr_bytes = need;
+  }
+  float* U = const_cast<float*>(td.U);
+  const float* A = U;                  // NULL source: the gradient directions were written into the subspace buffer itself
+  if (grads != nullptr && grads != td.U) {
+    if (src_is_host) {
+      const size_t bytes = static_cast<size_t>(td.rows) * td.rank * sizeof(float);
+      const int rc = check(ctx, cudaMemcpyAsync(U, grads, bytes, cudaMemcpyHostToDevice, st));
+      if (rc != ZGR_OK) return rc;
+    } else {
+      A = grads;
+    }
+  }
+  int* d_status = nullptr;
+  int rc = check(ctx, launch_build_subspace(A, td.rows, td.rank, U, ctx->d_qr, &d_status, nullptr, st));
+  if (rc != ZGR_OK) return rc;
+  ctx->launches += 6;
+  int status = 0;
+  rc = check(ctx, cudaMemcpyAsync(&status, d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (rc == ZGR_OK) rc = check(ctx, cudaStreamSynchronize(st));
+  if (rc != ZGR_OK) return rc;
+  if (status != 0) return ZGR_EINVAL;  // linearly dependent directions: nothing was written
+  // the new basis is in place: refresh the tensor-core operand copies exactly as for a delivered subspace
+  return zgr_update_subspace(ctx, tensor, nullptr, 0, stream);
 }
 
 int zgr_debug_plan(const zgr_tensor* tensors, int32_t n, const zgr_config* cfg, int32_t sm_count, int32_t tcgen05, int32_t multi,
@@ -771,6 +1045,7 @@ int zgr_update_subspaces(zgr_ctx* ctx, int32_t n, const int32_t* tensors, const 
     n_umma += ctx->descs[static_cast<size_t>(l)].umma ? 1 : 0;
   }
   if (ctx->sticky) return ctx->sticky;
+  if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   if (!ctx->ledger.empty()) return ZGR_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // every tensor of the tcgen05 path is listed: their operand copies are rebuilt by one launch after the copies
@@ -795,7 +1070,7 @@ int zgr_update_subspaces(zgr_ctx* ctx, int32_t n, const int32_t* tensors, const 
     }
     if (td.umma && !fused) {
       const int64_t rows_pad = ((td.rows + 127) / 128) * 128;
-      const int rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.Uhi, td.Ulo, st));
+      const int rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.ushift, td.Uhi, td.Ulo, st));
       if (rc != ZGR_OK) return rc;
       ctx->launches++;
     }
@@ -875,6 +1150,10 @@ int zgr_get_state(const zgr_ctx* ctx, int32_t* active, uint64_t* seed, double* n
   return ZGR_OK;
 }
 
+int zgr_debug_check_device(int32_t ctx_device, int32_t current_device) {
+  return (ctx_device >= 0 && ctx_device == current_device) ? ZGR_OK : ZGR_EINVAL;
+}
+
 int64_t zgr_launch_count(const zgr_ctx* ctx) { return ctx ? ctx->launches : -1; }
 
 void zgr_destroy(zgr_ctx* ctx) {
@@ -885,6 +1164,7 @@ void zgr_destroy(zgr_ctx* ctx) {
         cudaEventDestroy(ev.first);
         cudaEventDestroy(ev.second);
       }
+  for (cudaEvent_t e : ctx->layer_events) cudaEventDestroy(e);
   for (void* p : ctx->owned) cudaFree(p);
   delete ctx;
 }

@@ -13,8 +13,8 @@ PhiloxKeys host_make_keys(uint64_t seed);
 NormalScale host_make_scale(double s, int bits);
 
 // Read-only view of a context: descriptor of tensor l (host mirror), mixing scalars, generator mode,
-// sticky error code.  Returns false if ctx is null or l is out of range.
-bool host_ctx_view(const zgr_ctx* ctx, int32_t l, TensorDesc* desc, double* a, double* b, int* bits, int* sticky);
+// sticky error code, device ordinal the context is bound to.  Returns false if ctx is null or l is out of range.
+bool host_ctx_view(const zgr_ctx* ctx, int32_t l, TensorDesc* desc, double* a, double* b, int* bits, int* sticky, int* device);
 
 }  // namespace zgr
 #endif  // ZGR_HOST_INTERNAL_H_

@@ -12,7 +12,7 @@ struct TensorDesc {
   const float* U;        // rows x rank fp32 (caller's), or null
   const uint4* Ufrag;    // library-owned copy of U, split into bf16 hi/lo and laid out in the
                          // register order of the m16n8k16 A operand (tensor-core path only)
-  const int8_t* q;       // DTC codes rank x cols (int8), or rank rows of (cols+1)/2 bytes holding two unsigned
+  const int8_t* q;       // DTC codes qrows x cols (int8), or qrows rows of (cols+1)/2 bytes holding two unsigned
                          // 4-bit codes each, even column in the low nibble; null -> coefficients drawn from the seed
   const float* qscale;   // rank
   const float* qzero;    // rank or null
@@ -22,8 +22,10 @@ struct TensorDesc {
   int32_t id;            // generator tensor id (third counter word)
   int32_t dtype;
   int32_t qbits;         // 8 or 4: width of the codes behind q
+  int32_t qrows;         // rows of G taken from the codes (Sec. 3.4, proportion omega); rows beyond it are drawn from the seed
   int32_t umma;          // 1: served by the tcgen05 + TMA kernel (tensor maps and row-major hi/lo copies of U exist)
-  void* Uhi;             // library-owned, rows_pad x kpad bf16 row-major (TMA source), or null
+  int32_t ushift;        // the hi/lo copies hold U * 2^ushift (brings a typical entry of an orthonormal U near 1)
+  void* Uhi;             // library-owned, rows_pad x kpad fp16 row-major (TMA source), or null
   void* Ulo;
 };
 
@@ -72,6 +74,9 @@ struct SweepParams {
   const WorkItem* items;
   int32_t n_items;
   double* stats;         // 3 doubles per tensor (stats kernels only)
+  float* zout;           // rows x cols fp32 image of the one tensor swept (test hook of the tcgen05 kernel only)
+  int32_t kshift;        // tcgen05 kernel: the coefficient strips are scaled by a power of two so that sum_q |c_q| b 2^kshift
+                         // is near 1 (see the operand precision note in zgr_umma.cu)
 };
 
 }  // namespace zgr

@@ -18,6 +18,8 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
+
 #include "zgr_device.cuh"
 #include "zgr_kernels.h"
 
@@ -405,32 +407,36 @@ __global__ void split_subspace_kernel(const float* __restrict__ U, int64_t rows,
   out[idx] = make_uint4(regs[0], regs[1], regs[2], regs[3]);
 }
 
-// U (rows x r fp32) -> two row-major bf16 matrices (hi, lo), rows padded to a multiple of 128 and
-// columns to KP with zeros: the TMA source of the A operand.
-__global__ void split_subspace_rowmajor_kernel(const float* __restrict__ U, int64_t rows, int r, int kp, int64_t rows_pad,
-                                               __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+// U (rows x r fp32) -> two row-major fp16 matrices (hi, lo) holding U * 2^shift, rows padded to a multiple of
+// 128 and columns to KP with zeros: the TMA source of the A operand of the tcgen05 kernel.  hi + lo carries
+// 22 significant bits as long as the scaled entry is not far below 1 (lo must stay a normal fp16 number).
+__device__ __forceinline__ void split_f16_scaled(float x, float scale, __half& hi, __half& lo) {
+  const float y = x * scale;                       // power of two: exact
+  hi = __float2half_rn(y);
+  lo = __float2half_rn(y - __half2float(hi));
+}
+
+__global__ void split_subspace_rowmajor_kernel(const float* __restrict__ U, int64_t rows, int r, int kp, int64_t rows_pad, float scale,
+                                               __half* __restrict__ hi, __half* __restrict__ lo) {
   const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
   if (idx >= rows_pad * kp) return;
   const int64_t row = idx / kp;
   const int k = static_cast<int>(idx % kp);
   const float x = (row < rows && k < r) ? U[row * r + k] : 0.0f;
-  const __nv_bfloat16 h = __float2bfloat16_rn(x);
-  hi[idx] = h;
-  lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
+  split_f16_scaled(x, scale, hi[idx], lo[idx]);
 }
 
 __global__ void split_subspace_rowmajor_all_kernel(const SplitJob* __restrict__ jobs) {
   const SplitJob j = jobs[blockIdx.y];
   const int64_t n = j.rows_pad * j.kp;
-  __nv_bfloat16* hi = static_cast<__nv_bfloat16*>(j.hi);
-  __nv_bfloat16* lo = static_cast<__nv_bfloat16*>(j.lo);
+  __half* hi = static_cast<__half*>(j.hi);
+  __half* lo = static_cast<__half*>(j.lo);
+  const float scale = __int_as_float((127 + j.shift) << 23);
   for (int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; idx < n; idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
     const int64_t row = idx / j.kp;
     const int k = static_cast<int>(idx % j.kp);
     const float x = (row < j.rows && k < j.r) ? j.U[row * j.r + k] : 0.0f;
-    const __nv_bfloat16 h = __float2bfloat16_rn(x);
-    hi[idx] = h;
-    lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
+    split_f16_scaled(x, scale, hi[idx], lo[idx]);
   }
 }
 
@@ -547,11 +553,11 @@ cudaError_t launch_split_subspace_rowmajor_all(const SplitJob* d_jobs, int n_job
   return cudaGetLastError();
 }
 
-cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st) {
+cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, int shift, void* hi, void* lo, cudaStream_t st) {
   const int64_t n = rows_pad * kp;
   const int block = 256;
   split_subspace_rowmajor_kernel<<<static_cast<unsigned>((n + block - 1) / block), block, 0, st>>>(
-      U, rows, r, kp, rows_pad, static_cast<__nv_bfloat16*>(hi), static_cast<__nv_bfloat16*>(lo));
+      U, rows, r, kp, rows_pad, std::ldexp(1.0f, shift), static_cast<__half*>(hi), static_cast<__half*>(lo));
   return cudaGetLastError();
 }
 

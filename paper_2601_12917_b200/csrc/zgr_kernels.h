@@ -30,8 +30,10 @@ cudaError_t launch_sweep(const KernelChoice& kc, const SweepParams& p, int grid,
 int umma_strip_cols(int kpad);
 size_t umma_smem_bytes(int kpad);
 cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
+// Test hook: the sweep kernel with its fp32 results diverted to p.zout (see the ZOUT parameter of the kernel).
+cudaError_t launch_debug_z_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
 cudaError_t launch_stats_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st);
-cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, void* hi, void* lo, cudaStream_t st);
+cudaError_t launch_split_subspace_rowmajor(const float* U, int64_t rows, int r, int kp, int64_t rows_pad, int shift, void* hi, void* lo, cudaStream_t st);
 // The same for a device-resident list of tensors in one launch (grid.y = job).
 struct SplitJob {
   const float* U;
@@ -39,6 +41,7 @@ struct SplitJob {
   void* lo;
   int64_t rows, rows_pad;
   int32_t r, kp;
+  int32_t shift;   // the copies hold U * 2^shift
 };
 cudaError_t launch_split_subspace_rowmajor_all(const SplitJob* d_jobs, int n_jobs, cudaStream_t st);
 

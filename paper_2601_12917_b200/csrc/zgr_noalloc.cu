@@ -26,6 +26,8 @@ constexpr int kNormThreads = 256;
 static __device__ __align__(256) double g_norm_partials[3 * ZGR_NOALLOC_MAX_TILES];
 
 // Device address of g_norm_partials per device ordinal; looked up on the first call on that device.
+// The table is filled without a lock: two host threads that make their first call on the same device at
+// the same time both look the address up and both store the same value.
 constexpr int kMaxDevices = 64;
 double* g_partials_addr[kMaxDevices] = {};
 
@@ -102,9 +104,9 @@ using namespace zgr;
 extern "C" int zgr_tensor_norms_noalloc(zgr_ctx* ctx, uint64_t seed, int32_t tensor, double* dev_out3, void* stream) {
   TensorDesc td;
   double a, b;
-  int bits, sticky;
+  int bits, sticky, ctx_device;
   if (!dev_out3 || (reinterpret_cast<uintptr_t>(dev_out3) & 7) != 0) return ZGR_EINVAL;
-  if (!host_ctx_view(ctx, tensor, &td, &a, &b, &bits, &sticky)) return ZGR_EINVAL;
+  if (!host_ctx_view(ctx, tensor, &td, &a, &b, &bits, &sticky, &ctx_device)) return ZGR_EINVAL;
   if (sticky) return sticky;
   const int64_t strips = (td.cols + kTileCols - 1) / kTileCols;
   const int64_t row_tiles = (td.rows + kTileRows - 1) / kTileRows;
@@ -112,6 +114,9 @@ extern "C" int zgr_tensor_norms_noalloc(zgr_ctx* ctx, uint64_t seed, int32_t ten
 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ZGR_ECUDA;
+  // The tensor's subspace and coefficient pointers belong to the context's device; the scratch address
+  // below belongs to the current one.  They must be the same device.
+  if (zgr_debug_check_device(ctx_device, dev) != ZGR_OK) return ZGR_EINVAL;
   if (g_partials_addr[dev] == nullptr) {
     // One-time set-up on this device: translate the symbol into a device address.  (The symbol's
     // name is only a host-side handle; passing it to a kernel directly would hand the GPU a host address.)

@@ -10,9 +10,14 @@
 //   * tcgen05.mma builds   D = theta + c b U G   in tensor memory (fp32):
 //       - "theta" enters through identity products  D[:, 16j:16j+16] = theta[:, 16j:16j+16] * I16
 //         with theta's own 16-bit tile as the A operand, which unpacks it to fp32 exactly, for free;
-//       - U G is accumulated on top as  Ulo Ghi + Uhi Glo + Uhi Ghi  (bf16 split operands,
-//         about 2^-16 relative error per term), the strip of c b G living in shared memory as the
-//         K-major B operand for all row tiles of a work item.
+//       - U G is formed first as  Ulo Ghi + Uhi Glo + Uhi Ghi  with fp16 split operands (hi + lo carries 22
+//         significant bits, against 16 for a bf16 split, whose representation error of 4.5e-6 relative was the
+//         whole error of z on this path).  fp16 has a narrow exponent range, so both operands are kept near 1
+//         by powers of two: the library's copy of U holds U 2^j (j from the tensor's row count), the strips hold
+//         c b G 2^(s-j), and the accumulator therefore holds 2^s c b U G.  The identity products that bring
+//         theta in come last and use the instruction's accumulator scaling,  D <- theta I + 2^-s D
+//         (s <= 15 is an immediate of the instruction), which removes the factor exactly and for free.
+//         The strips of c b G live in shared memory as the K-major B operand for all row tiles of a work item.
 //   * The epilogue warps, in two groups that take alternate tiles (32 rows x 64 columns per warp, 32 columns
 //     at a time), read D with tcgen05.ld (one row per thread), add the isotropic
 //     normals (Philox4x32-10 + Box-Muller in registers), round to the storage type and write the
@@ -37,6 +42,14 @@ namespace zgr {
 namespace {
 
 constexpr unsigned kStaggerNs = 800;
+// Sleep between two polls of a barrier: the single-thread roles (which run ahead of the epilogue and share
+// their schedulers with epilogue warps) and the epilogue warps themselves.
+#ifndef ZGR_ROLE_SLEEP_NS
+#define ZGR_ROLE_SLEEP_NS 64
+#endif
+#ifndef ZGR_EPI_SLEEP_NS
+#define ZGR_EPI_SLEEP_NS 0
+#endif
 constexpr unsigned long long kWaitLimitCycles = 4000000000ull;  // ~2 s at 2 GHz
 
 // ---------------------------------------------------------------------------------------------
@@ -75,7 +88,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   uint32_t polls = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (BACKOFF) __nanosleep(64);
+    if (BACKOFF) __nanosleep(ZGR_ROLE_SLEEP_NS);
+    else if (ZGR_EPI_SLEEP_NS > 0) __nanosleep(ZGR_EPI_SLEEP_NS);
     if ((++polls & 255u) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
@@ -138,6 +152,16 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t b
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// D <- A B + 2^-SC D  (the accumulator-scaling form of the instruction; SC in [0, 15] is an immediate)
+template <int SC>
+__device__ __forceinline__ void umma_scaled_d(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, 1, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p, %4;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "n"(SC)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -197,12 +221,17 @@ struct Pack16<__half> {
   }
 };
 
-__device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uint32_t& lo) {
-  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+// fp16 hi/lo split of a pair of floats, packed as f16x2 (first value in the low half)
+__device__ __forceinline__ void split_f16(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const __half2 h = __floats2half2_rn(x0, x1);
   hi = *reinterpret_cast<const uint32_t*>(&h);
-  const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __uint_as_float(hi << 16), x1 - __uint_as_float(hi & 0xFFFF0000u));
+  const float2 hf = __half22float2(h);
+  const __half2 l = __floats2half2_rn(x0 - hf.x, x1 - hf.y);
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
+
+// Accumulator scale of a tensor in this call: s = clamp(ushift + kshift, 0, 15) (see the operand precision note above)
+__device__ __forceinline__ int acc_shift(const TensorDesc& td, const SweepParams& p) { return min(max(td.ushift + p.kshift, 0), 15); }
 
 // Tile configuration per contraction width: compile-time parameters (-D...) whose defaults are the measured
 // optimum on B200.  TILE_N = 192 runs 24 epilogue warps on 128 x 192 tiles (three 64-column boxes);
@@ -278,7 +307,11 @@ struct TileCoord {
 // MULTI = true applies several (seed, coefficient) terms in the one pass: the coefficient strips of
 // the terms are summed before the split (U (sum_q c_q b G_q) is one product), the isotropic normals
 // are added term by term in the epilogue.
-template <typename T, int BITS, int KP, bool STATS = false, bool MULTI = false>
+// ZOUT = true is the test hook of this kernel: the same loads, products and epilogue arithmetic, but the fp32
+// result of every element (accumulator plus normals, before the rounding to the storage type) goes to
+// p.zout[row * cols + col] by plain stores and nothing is written back to the weights.  On a zeroed
+// weight image with coefficient 1 that is z itself as this kernel computes it.
+template <typename T, int BITS, int KP, bool STATS = false, bool MULTI = false, bool ZOUT = false>
 __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
                                                                      int* __restrict__ error) {
   using Cfg = UmmaCfg<KP>;
@@ -370,8 +403,10 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
             if (t >= S) {
               // the epilogue has written tile t-S into this stage: store it, then the stage is free
               if (!mbar_wait<true>(BAR_OUT(s), ((t / S) - 1) & 1, abort_flag, error, 1)) { ok = false; break; }
-              store_tile(s);
-              tma_wait_read0();
+              if (!ZOUT) {
+                store_tile(s);
+                tma_wait_read0();
+              }
             }
             const int col0 = static_cast<int>(w.col0) + NS * sub;
             const int ncols = min(NS, w.ncols - NS * sub);
@@ -387,7 +422,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       const int total = t;
       for (int v = (total > S ? total - S : 0); v < total && ok && !STATS; ++v) {
         if (!mbar_wait<true>(BAR_OUT(v % S), (v / S) & 1, abort_flag, error, 2)) { ok = false; break; }
-        store_tile(v % S);
+        if (!ZOUT) store_tile(v % S);
       }
       if (!ok) {
         // aborting: let the loads already issued land before the CTA gives up its shared memory
@@ -408,7 +443,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
     // ===================================== MMA issuer =====================================
     if (elect_one()) {
       const uint32_t idesc_id = make_idesc(Pack16<T>::kFmt, 16);
-      const uint32_t idesc_ug = make_idesc(1, NS);
+      const uint32_t idesc_ug = make_idesc(0, NS);          // fp16 operands
       const uint64_t desc_id = make_desc(smem_u32(ident), 32);
       // Descriptors differ only in their start-address field (bits 0-13, address >> 4), so every
       // operand below is one of these bases plus a small constant.
@@ -419,6 +454,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       bool ok = true;
       for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x, ++item_no) {
         const WorkItem w = p.items[it];
+        const int sh = acc_shift(p.tensors[w.tensor], p);
         if (!mbar_wait<true>(BAR_G, item_no & 1, abort_flag, error, 3)) break;
         tc_fence_after();
         const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
@@ -430,33 +466,53 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
           const uint64_t desc_ulo = desc_uhi + static_cast<uint64_t>(Cfg::U_BYTES >> 4);
           for (int sub = 0; sub < nsub; ++sub, ++t) {
             const int s = t % S, b = t % NACC;
-            if (!STATS && !mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
             if (t >= NACC && !mbar_wait<true>(BAR_ACC_EMPTY(b), ((t / NACC) - 1) & 1, abort_flag, error, 5)) { ok = false; break; }
             tc_fence_after();
             const uint64_t desc_theta = desc_theta0 + static_cast<uint64_t>((s * Cfg::THETA_BYTES) >> 4);
             const uint32_t d = tmem_base + static_cast<uint32_t>(b * NS);
             const int nbox = (min(NS, w.ncols - NS * sub) + 63) / 64;
-            // theta -> fp32, 16 columns at a time
-            if (!STATS) {
-#pragma unroll
-              for (int c = 0; c < NS / 64; ++c) {
-                if (c < nbox) {
-#pragma unroll
-                  for (int k = 0; k < 4; ++k)
-                    umma(d + static_cast<uint32_t>(64 * c + 16 * k), desc_theta + static_cast<uint64_t>((c * 16384 + 32 * k) >> 4), desc_id, idesc_id, 0u);
-                }
-              }
-            }
-            // + c b U G, split operands
+            // 2^s c b U G, split operands
             const uint64_t desc_ghi = desc_g0 + static_cast<uint64_t>((sub * 2 * Cfg::G_BYTES) >> 4);
             const uint64_t desc_glo = desc_ghi + static_cast<uint64_t>(Cfg::G_BYTES >> 4);
 #pragma unroll
             for (int k = 0; k < KP / 16; ++k)
-              umma(d, desc_ulo + static_cast<uint64_t>(2 * k), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, (STATS && k == 0) ? 0u : 1u);
+              umma(d, desc_ulo + static_cast<uint64_t>(2 * k), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, k == 0 ? 0u : 1u);
 #pragma unroll
             for (int k = 0; k < KP / 16; ++k) umma(d, desc_uhi + static_cast<uint64_t>(2 * k), desc_glo + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
 #pragma unroll
             for (int k = 0; k < KP / 16; ++k) umma(d, desc_uhi + static_cast<uint64_t>(2 * k), desc_ghi + static_cast<uint64_t>(2 * k), idesc_ug, 1u);
+            // theta last, 16 columns at a time:  D <- theta I + 2^-s D
+            if (!STATS) {
+              if (!mbar_wait<true>(BAR_FULL(s), (t / S) & 1, abort_flag, error, 4)) { ok = false; break; }
+              tc_fence_after();
+#define ZGR_THETA_IN(SC)                                                                                                   \
+  _Pragma("unroll") for (int c = 0; c < NS / 64; ++c) {                                                                    \
+    if (c < nbox) {                                                                                                        \
+      _Pragma("unroll") for (int k = 0; k < 4; ++k)                                                                        \
+          umma_scaled_d<SC>(d + static_cast<uint32_t>(64 * c + 16 * k), desc_theta + static_cast<uint64_t>((c * 16384 + 32 * k) >> 4), \
+                            desc_id, idesc_id);                                                                            \
+    }                                                                                                                      \
+  }
+              switch (sh) {
+                case 0: ZGR_THETA_IN(0) break;
+                case 1: ZGR_THETA_IN(1) break;
+                case 2: ZGR_THETA_IN(2) break;
+                case 3: ZGR_THETA_IN(3) break;
+                case 4: ZGR_THETA_IN(4) break;
+                case 5: ZGR_THETA_IN(5) break;
+                case 6: ZGR_THETA_IN(6) break;
+                case 7: ZGR_THETA_IN(7) break;
+                case 8: ZGR_THETA_IN(8) break;
+                case 9: ZGR_THETA_IN(9) break;
+                case 10: ZGR_THETA_IN(10) break;
+                case 11: ZGR_THETA_IN(11) break;
+                case 12: ZGR_THETA_IN(12) break;
+                case 13: ZGR_THETA_IN(13) break;
+                case 14: ZGR_THETA_IN(14) break;
+                default: ZGR_THETA_IN(15) break;
+              }
+#undef ZGR_THETA_IN
+            }
             umma_commit(BAR_ACC_FULL(b));
           }
           if (ok) umma_commit(BAR_U_FREE(u));   // arrives once every product that reads this U tile has completed
@@ -485,6 +541,8 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
       const uint32_t tid = static_cast<uint32_t>(td.id);
       const int r = td.rank;
       const uint64_t tcols = static_cast<uint64_t>(td.cols);   // kept in a register: the barriers below force reloads of anything read through td
+      const int sh = acc_shift(td, p);
+      const float gscale = __int_as_float((127 + sh - td.ushift) << 23);   // 2^(s - j): the strips hold c b G 2^(s - j)
       if (GROUPS > 1 && t > 0) {
         // The strips are about to be overwritten.  With two groups this warp may be one tile ahead of the
         // other group, whose last tile of the previous item can still have products in flight that read the
@@ -518,7 +576,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           uint32_t hi, lo;
-          split_bf16(g0[i], g1[i], hi, lo);
+          split_f16(g0[i] * gscale, g1[i] * gscale, hi, lo);
           const uint32_t off = swizzle(static_cast<uint32_t>(((cc % NS) + i) * ROWB + 4 * kp), ROWB);
           sts32(g_hi + off, hi);
           sts32(g_lo + off, lo);
@@ -561,6 +619,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
             tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 16), h1);
             tmem_ld_wait();
             if constexpr (STATS) {
+              const float descale = __int_as_float((127 - sh) << 23);
               float f_iso = 0.0f, f_gd = 0.0f, f_z = 0.0f;
 #pragma unroll
               for (int o = 0; o < 4; ++o) {
@@ -572,7 +631,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
                 const bool live = row < row_end && NS * sub + 32 * cgrp + 8 * o < w.ncols;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                  const float gd = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
+                  const float gd = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]) * descale;   // no identity product here: undo 2^s
                   if (live) {
                     f_iso = fmaf(zi[i], zi[i], f_iso);
                     f_gd = fmaf(gd, gd, f_gd);
@@ -597,9 +656,18 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
                 for (int q = 1; q < p.n_terms; ++q)
                   normals8_acc<BITS>(p.term[q].keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.term[q].iso, acc);
               }
-              const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
-                                         Pack16<T>::pack(acc[6], acc[7]));
-              sts128(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4), q);
+              if constexpr (ZOUT) {
+                const int col = NS * sub + 32 * cgrp + 8 * o;          // within the item's strip
+                if (row < row_end && col < w.ncols) {
+                  float4* dst = reinterpret_cast<float4*>(p.zout + static_cast<uint64_t>(row) * tcols + static_cast<uint64_t>(w.col0 + col));
+                  dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                  dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                }
+              } else {
+                const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
+                                           Pack16<T>::pack(acc[6], acc[7]));
+                sts128(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4), q);
+              }
             }
             }
           }
@@ -644,11 +712,11 @@ size_t umma_smem_bytes(int kpad) {
 int umma_strip_cols(int kpad) { return kpad == 64 ? UmmaCfg<64>::NS * UmmaCfg<64>::NSUB : (kpad == 32 ? UmmaCfg<32>::NS * UmmaCfg<32>::NSUB : UmmaCfg<16>::NS * UmmaCfg<16>::NSUB); }
 
 namespace {
-template <typename T, int BITS, bool STATS = false, bool MULTI = false>
+template <typename T, int BITS, bool STATS = false, bool MULTI = false, bool ZOUT = false>
 cudaError_t launch_umma_kp(int kpad, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
 #define ZGR_LAUNCH_UMMA(KPV)                                                                                       \
   {                                                                                                                \
-    auto k = sweep_umma_kernel<T, BITS, KPV, STATS, MULTI>;                                                               \
+    auto k = sweep_umma_kernel<T, BITS, KPV, STATS, MULTI, ZOUT>;                                                         \
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<KPV>::SMEM_BYTES); \
     if (e != cudaSuccess) return e;                                                                                \
     k<<<grid, UmmaCfg<KPV>::THREADS, UmmaCfg<KPV>::SMEM_BYTES, st>>>(p, tmaps, error);                                      \
@@ -675,6 +743,17 @@ cudaError_t launch_umma_typed(const KernelChoice& kc, const SweepParams& p, cons
 cudaError_t launch_sweep_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
   if (kc.dtype == 2) return launch_umma_typed<__nv_bfloat16>(kc, p, tmaps, error, grid, st);
   if (kc.dtype == 1) return launch_umma_typed<__half>(kc, p, tmaps, error, grid, st);
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_debug_z_umma(const KernelChoice& kc, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
+  if (p.zout == nullptr || p.n_terms != 1) return cudaErrorInvalidValue;
+  if (kc.dtype == 2)
+    return kc.bits == 32 ? launch_umma_kp<__nv_bfloat16, 32, false, false, true>(kc.kpad, p, tmaps, error, grid, st)
+                         : launch_umma_kp<__nv_bfloat16, 16, false, false, true>(kc.kpad, p, tmaps, error, grid, st);
+  if (kc.dtype == 1)
+    return kc.bits == 32 ? launch_umma_kp<__half, 32, false, false, true>(kc.kpad, p, tmaps, error, grid, st)
+                         : launch_umma_kp<__half, 16, false, false, true>(kc.kpad, p, tmaps, error, grid, st);
   return cudaErrorInvalidValue;
 }
 

@@ -68,6 +68,14 @@ def lib() -> ctypes.CDLL:
         L.zgr_get_stats.argtypes = [vp, u64, ctypes.POINTER(dbl), vp]
         L.zgr_debug_philox.argtypes = [vp, u64, i32, i32, u64, i64, vp, vp]
         L.zgr_debug_z.argtypes = [vp, u64, i32, vp, vp]
+        L.zgr_debug_z_tcgen05.argtypes = [vp, u64, i32, vp, vp]
+        L.zgr_debug_z_tcgen05.restype = ctypes.c_int
+        L.zgr_debug_check_device.argtypes = [i32, i32]
+        L.zgr_debug_check_device.restype = ctypes.c_int
+        L.zgr_adapt_alpha.argtypes = [vp, ctypes.POINTER(dbl), dbl, dbl, dbl, ctypes.POINTER(dbl)]
+        L.zgr_adapt_alpha.restype = ctypes.c_int
+        L.zgr_build_subspace.argtypes = [vp, i32, vp, i32, vp]
+        L.zgr_build_subspace.restype = ctypes.c_int
         L.zgr_get_scalars.argtypes = [vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
         L.zgr_get_state.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(u64), ctypes.POINTER(dbl)]
         L.zgr_update_subspace.argtypes = [vp, i32, vp, i32, vp]
@@ -170,6 +178,28 @@ class Zgr:
         """New mixing ratio for the following steps (zgr_set_alpha)."""
         _check(lib().zgr_set_alpha(self._h, alpha), "zgr_set_alpha")
 
+    def adapt_alpha(self, stats, alpha_min: float = 0.05, alpha_max: float = 0.95, eta: float = 1.0) -> float:
+        """Move the mixing ratio towards the balance of the two parts' energies (zgr_adapt_alpha); `stats` is
+        the array returned by get_stats under the current ratio.  Returns the new ratio."""
+        import numpy as np
+        st = np.ascontiguousarray(stats, dtype=np.float64).reshape(-1)
+        assert st.size == 3 * self.n
+        out = ctypes.c_double()
+        _check(lib().zgr_adapt_alpha(self._h, st.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), alpha_min, alpha_max, eta, ctypes.byref(out)),
+               "zgr_adapt_alpha")
+        return out.value
+
+    def build_subspace(self, tensor: int, grads=None, stream=None) -> None:
+        """Orthonormal basis of the span of the gradient directions `grads` (rows x rank fp32 torch tensor on the
+        host or on the device; None if they were written into the subspace buffer) becomes the subspace of
+        `tensor` (zgr_build_subspace)."""
+        if grads is None:
+            ptr, host = None, 0
+        else:
+            assert grads.is_contiguous() and grads.dtype == self._keep[1][tensor].dtype and grads.shape == self._keep[1][tensor].shape
+            ptr, host = grads.data_ptr(), 0 if grads.is_cuda else 1
+        _check(lib().zgr_build_subspace(self._h, tensor, ptr, host, _stream_ptr(stream)), "zgr_build_subspace")
+
     # -- compressed coefficients ----------------------------------------------------------------
     def set_coeffs_dtc(self, tensor: int, q, scale, zero=None, bits: int = 8) -> None:
         self._keep.append((q, scale, zero))
@@ -240,6 +270,14 @@ class Zgr:
         w = self._keep[0][tensor]
         out = torch.empty(w.shape, dtype=torch.float32, device=w.device)
         _check(lib().zgr_debug_z(self._h, seed, tensor, out.data_ptr(), _stream_ptr(stream)), "zgr_debug_z")
+        return out
+
+    def debug_z_tcgen05(self, seed: int, tensor: int, stream=None):
+        """z of `tensor` in fp32 as the tcgen05 sweep kernel itself computes it (zgr_debug_z_tcgen05)."""
+        import torch
+        w = self._keep[0][tensor]
+        out = torch.empty(w.shape, dtype=torch.float32, device=w.device)
+        _check(lib().zgr_debug_z_tcgen05(self._h, seed, tensor, out.data_ptr(), _stream_ptr(stream)), "zgr_debug_z_tcgen05")
         return out
 
     def device_status(self) -> int:

@@ -10,7 +10,12 @@ Tolerances (stated by the benchmark spec, derived in the design notes):
     |c| sigma_z, sigma_z = sqrt(a^2 + b^2 r/m) being the rms size of z in that tensor (where
     theta + c z cancels, the ulp of the tiny result is below the resolution of the fp32 arithmetic
     that its operands went through).
-Each check also reports how many elements moved at all, so that a sweep that does nothing cannot pass.
+Each check also reports how many elements moved at all, so that a sweep that does nothing cannot pass,
+and the strict statistics of 16-bit results: the bit-identical fraction, the fraction that differs by more
+than one ulp OF THE ORACLE'S RESULT (the elements that need the wider reading above) and the worst such
+difference.  The bit-identical fraction is held against what the claimed accuracy of z allows: an error of
+at most delta in z moves theta + c z by at most |c| delta, which crosses a rounding boundary of the result
+with probability |c| delta / ulp(result); three times the mean of that over the elements is the allowance.
 """
 from __future__ import annotations
 
@@ -48,21 +53,42 @@ def ulp(x: np.ndarray, dtype: str) -> np.ndarray:
     return 2.0 ** (np.floor(np.log2(ax)) - (SIG_BITS[dtype] - 1))
 
 
+# Claimed absolute accuracy of a unit-variance z on the 16-bit kernel families (hardware-approximation
+# Gaussian transform; fp16-split tensor-core contraction above rank 8).  test_gpu_tcgen05_z.py and
+# test_perturbation_matches_oracle measure it (at most 9e-6 seen); the bit-identical allowance below is derived from it.
+DELTA_Z_16BIT = 1e-5
+
+STATS_LOG = []   # one entry per 16-bit check of this process; summarised at the end of the session (conftest.py)
+
+
 def check_sweep(got: np.ndarray, exp: np.ndarray, before: np.ndarray, dtype: str, theta_max: float, what: str = "",
-                operand: float = 0.0) -> dict:
-    """Assert the per-call tolerance; returns a small report."""
+                operand: float = 0.0, c_abs: float = None, z_scale: float = 1.0) -> dict:
+    """Assert the per-call tolerance; returns a small report.  c_abs = |c| of the call (sum of |c_q| for several
+    terms) switches the bit-identical allowance on; z_scale = size of a unit of z (1 in the unit normalisation)."""
     diff = np.abs(got - exp)
+    rep = {"equal": float(np.mean(got == exp)) if got.size else 1.0, "moved": float(np.mean(exp != before)) if got.size else 0.0,
+           "max_abs": float(diff.max()) if diff.size else 0.0, "n": int(got.size)}
     if dtype == "f32":
         tol = 1e-6 * theta_max
         worst = float(diff.max()) if diff.size else 0.0
         assert worst <= tol, f"{what}: fp32 max-abs error {worst:.3e} > {tol:.3e}"
-    else:
-        u = ulp(np.maximum(np.maximum(np.abs(before), np.abs(exp)), operand), dtype)
-        bad = diff > u
-        assert not bad.any(), (f"{what}: {int(bad.sum())} of {bad.size} elements differ by more than 1 ulp; "
-                               f"worst {float((diff / u).max()):.2f} ulp")
-    return {"equal": float(np.mean(got == exp)) if got.size else 1.0, "moved": float(np.mean(exp != before)) if got.size else 0.0,
-            "max_abs": float(diff.max()) if diff.size else 0.0}
+        return rep
+    u = ulp(np.maximum(np.maximum(np.abs(before), np.abs(exp)), operand), dtype)
+    bad = diff > u
+    assert not bad.any(), (f"{what}: {int(bad.sum())} of {bad.size} elements differ by more than 1 ulp; "
+                           f"worst {float((diff / u).max()):.2f} ulp")
+    if got.size:
+        us = ulp(exp, dtype)                                  # strict: the ulp of the oracle's own result
+        strict = diff / us
+        rep.update(strict_beyond_1ulp=float(np.mean(strict > 1.0)), strict_worst_ulp=float(strict.max()),
+                   needs_wide=int(np.sum(strict > 1.0)))
+        if c_abs is not None:
+            allowed = 3.0 * float(np.mean(np.minimum(1.0, c_abs * DELTA_Z_16BIT * z_scale / us))) + 5.0 / got.size
+            rep["allowed_unequal"] = allowed
+            assert 1.0 - rep["equal"] <= allowed, (f"{what}: {100 * (1 - rep['equal']):.3f} % of the results are not bit-identical to the "
+                                                   f"oracle's; a z accurate to {DELTA_Z_16BIT:g} allows {100 * allowed:.3f} %")
+        STATS_LOG.append((what, rep))
+    return rep
 
 
 class Pair:
@@ -124,8 +150,13 @@ class Pair:
         for l, t in enumerate(ots):
             got = to_double(self.theta[l])
             reports.append(check_sweep(got, exps[l], before[l], self.dtype, theta_max,
-                                       f"{what} tensor {l} {self.shapes[l]} r={self.ranks[l]}", operand=abs(c) * self.sigma_z(l)))
+                                       f"{what} tensor {l} {self.shapes[l]} r={self.ranks[l]}", operand=abs(c) * self.sigma_z(l),
+                                       c_abs=abs(c), z_scale=self.z_unit()))
         return reports
+
+    def z_unit(self) -> float:
+        """Size of one unit of z: 1 in the unit normalisation, 1/sqrt(d) in the paper's."""
+        return 1.0 if self.scale_mode == zgr.SCALE_UNIT else 1.0 / float(np.sqrt(self.d))
 
     def call_and_check_multi(self, seeds, coeffs, fn, what: str):
         """Run one library call `fn()` that applies sum_q coeffs[q] z(seeds[q]); the oracle starts from the same theta."""
@@ -143,7 +174,8 @@ class Pair:
         for l, t in enumerate(ots):
             got = to_double(self.theta[l])
             reports.append(check_sweep(got, exps[l], before[l], self.dtype, theta_max,
-                                       f"{what} tensor {l} {self.shapes[l]} r={self.ranks[l]}", operand=operand * self.sigma_z(l)))
+                                       f"{what} tensor {l} {self.shapes[l]} r={self.ranks[l]}", operand=operand * self.sigma_z(l),
+                                       c_abs=operand, z_scale=self.z_unit()))
         return reports
 
     def sigma_z(self, l: int) -> float:

@@ -43,6 +43,18 @@ def test_error_strings_and_null_arguments():
     L.zgr_destroy(None)
 
 
+def test_current_device_check_of_the_launching_calls():
+    # Every call that enqueues work compares the context's device with the current one through this host-only
+    # function and returns ZGR_EINVAL on a mismatch, before anything is launched (a context's tables, tensor
+    # maps and borrowed pointers are addresses of its own device).
+    L = zgr.lib()
+    assert L.zgr_debug_check_device(0, 0) == zgr.OK
+    assert L.zgr_debug_check_device(3, 3) == zgr.OK
+    assert L.zgr_debug_check_device(0, 1) == zgr.EINVAL
+    assert L.zgr_debug_check_device(1, 0) == zgr.EINVAL
+    assert L.zgr_debug_check_device(-1, -1) == zgr.EINVAL       # no valid device was current at zgr_init
+
+
 def test_argument_validation_happens_before_any_device_work():
     L = zgr.lib()
     h = ctypes.c_void_p()

@@ -26,6 +26,10 @@ def test_worked_scalars_of_the_smallest_configuration():
     assert g == pytest.approx(v["g"], rel=1e-12)
     assert v["lr"] * g == pytest.approx(v["lr_times_g"], rel=1e-12)
     assert abs(v["eps"] - v["lr"] * g) < 1e-15                      # vanishes up to the rounding of the decimal inputs
+    # the fused restore + update coefficient: with -eps still applied it cancels, on the server side (nothing
+    # applied) it is the bare step -lr g
+    assert abs(oracle.update_coefficient(-v["eps"], v["loss_plus"], v["loss_minus"], v["eps"], v["lr"])) < 1e-15
+    assert oracle.update_coefficient(0.0, v["loss_plus"], v["loss_minus"], v["eps"], v["lr"]) == pytest.approx(-v["lr_times_g"], rel=1e-12)
     d, K = int(v["d"]), int(v["K"])
     assert d == 4 * 256 * 256 + 4 * 256 and K == 4 * 4 * 256
     a, b = oracle.mix_scalars(0.5, d, K, oracle.SCALE_PAPER)

@@ -55,7 +55,10 @@ Z_CASES = [
 # absolute tolerance on a unit-variance z: fp32 tensors use the accurate transform and an exact fp32
 # contraction; 16-bit tensors use the hardware approximations and, above rank 8, split-bf16 tensor cores
 Z_TOL = {("f32", "iso"): 2e-6, ("f32", "fma"): 2e-6, ("f32", "mma"): 3e-6, ("f32", "generic"): 3e-6,
-         ("bf16", "iso"): 1e-5, ("bf16", "fma"): 1e-5, ("bf16", "mma"): 1e-4, ("bf16", "generic"): 1e-5}
+         ("bf16", "iso"): 1e-5, ("bf16", "fma"): 1e-5, ("bf16", "mma"): 4e-5, ("bf16", "generic"): 1e-5}
+# ("mma" rows: zgr_debug_z runs the legacy mma.sync kernel for these tensors, whose operands are split into bf16
+#  hi/lo (16 significant bits: 4.5e-6 rms, up to 4e-5 in the tail); the tcgen05 kernel that the sweeps use for them
+#  splits into fp16 hi/lo and is compared with the oracle at 1.2e-5 in test_gpu_tcgen05_z.py)
 
 
 @pytest.mark.parametrize("bits", [32, 16])
@@ -109,8 +112,8 @@ def test_step_per_call_parity(model, dtype, bits):
     for call in reports:
         for rep in call:
             assert rep["moved"] > 0.3, rep         # the sweep really changed the weights
-            if dtype != "f32":
-                assert rep["equal"] > 0.9, rep     # and almost every 16-bit result is bit-identical to the oracle
+            # (16-bit results: check_sweep holds the bit-identical fraction against what a z accurate to
+            #  helpers.DELTA_Z_16BIT allows for this call's coefficient)
     assert p.lib.state()[0] is False
 
 
@@ -314,6 +317,6 @@ def test_many_work_items_per_block(dtype, rows, cols, rank):
     p = Pair([(rows, cols)], [rank], dtype, bits=16, seed=21)
     reports = p.step(seed=12, lp=2.3, lm=1.8, lr=1e-4)
     for call in reports:
-        assert call[0]["moved"] > 0.3 and call[0]["equal"] > 0.9, call
+        assert call[0]["moved"] > 0.3 and call[0]["equal"] > 0.98, call
     seeds, coeffs = [31, 32], [1e-3, -7e-4]
     p.call_and_check_multi(seeds, coeffs, lambda: p.lib.sweep_multi(seeds, coeffs), "sweep_multi")

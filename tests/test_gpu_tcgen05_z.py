@@ -1,0 +1,108 @@
+"""z of the tcgen05 sweep kernel itself, element by element against the oracle (needs a B200).
+
+zgr_debug_z runs 16-bit tensors of rank > 8 through the legacy mma.sync kernel (it sweeps an fp32 image,
+which the tcgen05 kernel cannot read), so it says nothing about the kernel that carries the OPT- and
+LLaMA-shaped configurations.  zgr_debug_z_tcgen05 runs that kernel (TMA loads of a zeroed 16-bit image,
+identity products, the three split-bf16 products of U G, tensor-memory reads, generator and Gaussian
+transform in the epilogue) and hands back its fp32 result before the rounding to the storage type.
+
+Bounds (absolute, z of unit variance):
+  * whole z:        1.2e-5 at most and 1.5e-6 rms.  Measured: 3e-6 .. 9e-6 at most, 8.1e-7 rms, the same for every
+                    rank, storage type and generator mode: the hardware-approximation transform (lg2/sqrt/sin/cos on a
+                    radius of at most 4.85) and the fp16-split contraction contribute about equally.  With operands
+                    split into bf16 hi/lo, as in the first version of the kernel, the same test read 2.6e-5 at most and
+                    3.2e-6 rms (the representation error of a 16-bit significand); a dropped low-order product, or a
+                    single 16-bit operand, costs 2^-9 .. 2^-12 relative of the guided part, i.e. 2e-4 .. 1e-3: twenty
+                    to a hundred times the bound.
+  * guided part alone (alpha = 0, so a = 0 and the normals vanish): the same bound relative to its rms size,
+    which isolates the contraction from the transform.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_12917_b200 import zgr
+
+from helpers import Pair, to_double
+
+pytestmark = pytest.mark.gpu
+
+# (shape, rank): contraction widths 16, 32 and 64, ranks that are padded up to them, a ragged last strip
+# (columns not a multiple of the 128-column tile nor of the strip), a ragged last row block (rows not a
+# multiple of 128), several work items per tensor, and a tensor with fewer rows than one row block.
+CASES = [
+    ((300, 392), 16), ((130, 1032), 16), ((48, 128), 12),
+    ((300, 392), 32), ((200, 512), 32), ((384, 264), 24),
+    ((130, 1032), 64), ((96, 520), 64), ((72, 64), 40),
+]
+Z_BOUND = 1.2e-5
+Z_RMS_BOUND = 1.5e-6
+
+
+@pytest.mark.parametrize("bits", [16, 32])
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+@pytest.mark.parametrize("shape,rank", CASES)
+def test_tcgen05_kernel_z_matches_oracle(shape, rank, dtype, bits):
+    p = Pair([shape, (1, 40)], [rank, 0], dtype, bits=bits, seed=3)
+    seed = 7654321
+    got = to_double(p.lib.debug_z_tcgen05(seed, 0))
+    assert p.lib.device_status() == 0
+    z, iso, gd = oracle.z_tensor(p.oracle_tensor(0), seed, 0, bits, p.a, p.b, parts=True)
+    err = np.abs(got - z.ravel())
+    rel_guided = err.max() / np.sqrt(np.mean(gd**2))
+    print(f"tcgen05 z {shape} r={rank} {dtype} bits={bits}: max |z_gpu - z_oracle| = {err.max():.3e}, rms {np.sqrt(np.mean(err**2)):.3e} "
+          f"(guided rms {np.sqrt(np.mean(gd**2)):.3f}, max error / guided rms = {rel_guided:.3e})")
+    assert err.max() <= Z_BOUND, f"{shape} r={rank} {dtype}: max |z_gpu - z_oracle| = {err.max():.3e}"
+    assert np.sqrt(np.mean(err**2)) <= Z_RMS_BOUND
+    assert np.abs(z).max() > 2.0 and np.sqrt(np.mean(gd**2)) > 0.3     # both parts are really there
+    # a tensor that the tcgen05 kernel does not serve is refused, not silently routed elsewhere
+    with pytest.raises(zgr.ZgrError) as e:
+        p.lib.debug_z_tcgen05(seed, 1)
+    assert e.value.code == zgr.ESTATE
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+@pytest.mark.parametrize("shape,rank", [((300, 392), 16), ((300, 392), 32), ((130, 1032), 64)])
+def test_tcgen05_kernel_guided_part_alone(shape, rank, dtype):
+    # alpha = 0: a = 0, every normal is multiplied by zero and z = b U G exactly as the tensor cores form it
+    p = Pair([shape], [rank], dtype, bits=16, seed=5, alpha=0.0)
+    seed = 99
+    got = to_double(p.lib.debug_z_tcgen05(seed, 0))
+    z, iso, gd = oracle.z_tensor(p.oracle_tensor(0), seed, 0, 16, p.a, p.b, parts=True)
+    assert np.all(iso == 0)
+    err = np.abs(got - gd.ravel())
+    rms = np.sqrt(np.mean(gd**2))
+    print(f"tcgen05 guided part {shape} r={rank} {dtype}: max error {err.max():.3e}, rms error {np.sqrt(np.mean(err**2)):.3e}, guided rms {rms:.3f}")
+    assert err.max() <= Z_BOUND * max(1.0, rms)
+    # in span(U): the component of z outside the subspace vanishes (Eq. (perturbation) with alpha = 0)
+    U = p.U[0].cpu().numpy().astype(np.float64)
+    G = got.reshape(shape)
+    resid = G - U @ (U.T @ G)
+    assert np.abs(resid).max() <= 5e-5 * max(1.0, rms)
+
+
+def test_tcgen05_kernel_z_with_compressed_coefficients():
+    # the DTC form of the coefficients (Sec. 3.4) through the same kernel: int8 codes, then packed INT4 codes
+    from paper_2601_12917_b200 import synth
+    shape, rank = (260, 520), 64
+    p = Pair([shape], [rank], "bf16", bits=16, seed=8)
+    q, sc = synth.dtc_payload(rank, shape[1], seed=2)
+    p.set_dtc(0, q, sc)
+    got = to_double(p.lib.debug_z_tcgen05(11, 0))
+    exp = oracle.z_tensor(p.oracle_tensor(0), 11, 0, 16, p.a, p.b).ravel()
+    assert np.abs(got - exp).max() <= Z_BOUND
+    G = oracle.coeffs(9, 0, 16, rank, shape[1])
+    q4, sc4, ze4 = oracle.dtc_quantise_int4(G)
+    p.set_dtc(0, q4, sc4, ze4, bits=4)
+    got = to_double(p.lib.debug_z_tcgen05(11, 0))
+    exp = oracle.z_tensor(p.oracle_tensor(0), 11, 0, 16, p.a, p.b).ravel()
+    assert np.abs(got - exp).max() <= Z_BOUND
+
+
+def test_tcgen05_kernel_z_leaves_the_weights_alone():
+    p = Pair([(256, 256)], [32], "bf16", bits=16, seed=1)
+    before = p.theta[0].clone()
+    p.lib.debug_z_tcgen05(5, 0)
+    torch.cuda.synchronize()
+    assert torch.equal(before, p.theta[0]) and p.lib.state()[0] is False

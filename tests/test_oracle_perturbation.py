@@ -132,3 +132,35 @@ def test_parts_add_up_and_stats():
     np.testing.assert_allclose(gd, b * (t.U.astype(np.float64) @ G), atol=1e-14)
     st = oracle.stats_tensor(t, 1, 0, 32, a, b)
     np.testing.assert_allclose(st, [(iso**2).sum(), (gd**2).sum(), (z**2).sum()], rtol=1e-12)
+
+
+# ------------------------------------------------------------------------------------- a proportion of the coefficients compressed
+@pytest.mark.parametrize("qrows", [0, 1, 5, 8])
+def test_mixed_coefficient_source(qrows):
+    """Sec. 3.4, adaptive proportion: only part of the guided payload arrives compressed.  Here the first qrows
+    rows of G_l are dequantised codes, x = lambda (x_q - delta), the other rows are drawn from the seed.  Checked
+    against a dense construction from the two pure sources, and against them at the two ends."""
+    rows, cols, r, seed, tid, bits = 24, 40, 8, 77, 3, 32
+    U = synth.subspace(rows, r, 5)
+    q_full, sc_full = synth.dtc_payload(r, cols, seed=4)
+    ze_full = (np.arange(r) % 3 - 1).astype(np.float32)
+    a, b = 0.6, 1.7
+    t = oracle.OracleTensor(theta=np.zeros(rows * cols, dtype=np.float32), rows=rows, cols=cols, dtype=oracle.F32, U=U,
+                            q=q_full[:qrows], scale=sc_full[:qrows], zero=ze_full[:qrows])
+    z, iso, gd = oracle.z_tensor(t, seed, tid, bits, a, b, parts=True)
+    G_seed = oracle.coeffs(seed, tid, bits, r, cols)
+    G_code = oracle.dtc_dequantise(q_full, sc_full, ze_full)
+    G = np.vstack([G_code[:qrows], G_seed[qrows:]])
+    np.testing.assert_allclose(gd, b * (U.astype(np.float64) @ G), atol=1e-13)
+    np.testing.assert_allclose(oracle.coeffs(seed, tid, bits, r, cols, q_full[:qrows], sc_full[:qrows], ze_full[:qrows]), G, atol=0)
+    pure_seed = oracle.OracleTensor(theta=t.theta, rows=rows, cols=cols, dtype=oracle.F32, U=U)
+    pure_code = oracle.OracleTensor(theta=t.theta, rows=rows, cols=cols, dtype=oracle.F32, U=U, q=q_full, scale=sc_full, zero=ze_full)
+    if qrows == 0:
+        np.testing.assert_array_equal(z, oracle.z_tensor(pure_seed, seed, tid, bits, a, b))
+    if qrows == r:
+        np.testing.assert_array_equal(z, oracle.z_tensor(pure_code, seed, tid, bits, a, b))
+    # the random-access form and the norms see the same mixture
+    idx = np.arange(0, rows * cols, 7)
+    np.testing.assert_allclose(oracle.z_elements(t, seed, tid, bits, a, b, idx), z.ravel()[idx], atol=1e-14)
+    st = oracle.stats_tensor(t, seed, tid, bits, a, b)
+    np.testing.assert_allclose(st, [np.sum(iso**2), np.sum(gd**2), np.sum(z**2)], rtol=1e-13)
