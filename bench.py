@@ -271,6 +271,80 @@ def measure_other(name, device, bits, steps, peak, peak_kind):
     return out
 
 
+def layer_table(wl):
+    """Tensor index one past each layer: the embedding, every Transformer block, and what follows the last block."""
+    ends, prev, seen_block = [], None, False
+    for l, t in enumerate(wl.tensors):
+        prefix = t.name.split(".")[0]
+        is_block = prefix.startswith("l") and prefix[1:].isdigit()
+        seen_block = seen_block or is_block
+        key = prefix if is_block else ("after the blocks" if seen_block else "before the blocks")
+        if prev is not None and key != prev:
+            ends.append(l)
+        prev = key
+    ends.append(len(wl.tensors))
+    return ends
+
+
+def measure_overlap(device, bits):
+    """Sec. 3.3 / 3.4 on the DTC configuration: the compressed coefficients of layer l + 1 travel from pinned host
+    memory on a copy stream while layer l is swept (zgr_perturb_layers).  Reports the per-layer transmission time
+    T_t against the per-layer sweep time T_cc, and what the delivery adds to the sweep."""
+    import torch
+    from paper_2601_12917_b200 import synth, zgr
+    wl = synth.workload("llama_13b")
+    free, _ = torch.cuda.mem_get_info()
+    if free < wl.params * 2 * 1.3 + 4e9:
+        return {"workload": wl.name, "skipped": "not enough free device memory"}
+    dm = synth.materialise(wl, device, seed=0)
+    z = zgr.from_device_model(dm, bits)
+    ends = layer_table(wl)
+    deliveries = [(l, dm.q[l].cpu().pin_memory(), dm.scale[l].cpu().pin_memory(), None) for l in range(len(wl.tensors)) if dm.q[l] is not None]
+    payload = sum(q.numel() + 4 * sc.numel() for _, q, sc, _ in deliveries)
+    stream, copy_stream = torch.cuda.current_stream(), torch.cuda.Stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps=3):
+        fn(0)
+        z.restore_update(0, 2.0, 2.0, 0.0)
+        torch.cuda.synchronize()
+        total = 0.0
+        for i in range(reps):
+            ev0.record(stream)
+            fn(1 + i)
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            total += ev0.elapsed_time(ev1)
+            z.restore_update(1 + i, 2.0, 2.0, 0.0)
+        torch.cuda.synchronize()
+        return total / reps
+
+    one_launch = timed(lambda s: z.perturb(s, wl.eps))
+    layerwise = timed(lambda s: z.perturb_layers(s, wl.eps, ends, copy_stream=copy_stream))
+    delivered = timed(lambda s: z.perturb_layers(s, wl.eps, ends, deliveries, copy_stream=copy_stream))
+    # the transmission alone
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(copy_stream):
+        c0.record(copy_stream)
+        for l, q, sc, _ in deliveries:
+            dm.q[l].copy_(q, non_blocking=True)
+            dm.scale[l].copy_(sc, non_blocking=True)
+        c1.record(copy_stream)
+    torch.cuda.synchronize()
+    copy_ms = c0.elapsed_time(c1)
+    n_layers = len(ends)
+    out = {"workload": wl.name, "layers": n_layers, "omega": 1.0, "payload_bytes": payload, "transmission_ms": copy_ms,
+           "sweep_ms_one_launch_per_kernel": one_launch, "sweep_ms_layerwise": layerwise, "sweep_ms_layerwise_with_delivery": delivered,
+           "per_layer": {"T_t_ms": copy_ms / n_layers, "T_cc_ms": layerwise / n_layers},
+           "transmission_hidden": 1.0 - max(0.0, delivered - layerwise) / copy_ms,
+           "omega_that_still_hides": min(1.0, layerwise / copy_ms),
+           "what": "H2D of the int8 coefficients and scales of layer l+1 on a copy stream while layer l is swept; T_t <= T_cc per layer means the transmission is hidden"}
+    z.close()
+    del z, dm
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -387,7 +461,7 @@ def main():
                "ms_per_step": ms_e / n_e2e, "what": "subspaces H2D from pinned memory + step + per-tensor norms D2H, through the C ABI"}
 
     # ---- the other configurations, briefly (single process only; the headline above is unaffected) ----
-    others = None
+    others = overlap = None
     z.close()
     if world == 1 and not args.no_others and args.layers is None and wl.name == "llama_7b":
         del dm
@@ -396,6 +470,7 @@ def main():
         full = measure_other("llama_7b", device, 32, 3, peak, peak_kind)      # the headline workload with 32 random bits per normal
         full["bits_per_normal"] = 32
         others.append(full)
+        overlap = measure_overlap(device, args.bits)
 
     if rank == 0:
         sweeps = 3 * wl.queries if args.schedule == "sequential" else 2 * wl.queries + 1
@@ -408,7 +483,7 @@ def main():
                            "lr": wl.lr, "scale_mode": "unit", "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only"},
                 "sweep_params_per_s": value * sweeps, "hbm_gbs_all_sweeps": value * sweeps * 2 * eb / 1e9,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-                "kernels": kernels, "other_configs": others}
+                "kernels": kernels, "other_configs": others, "overlap": overlap}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -31,6 +31,10 @@ class ZgrConfig(ctypes.Structure):
     _fields_ = [("alpha", ctypes.c_double), ("eps", ctypes.c_double), ("scale_mode", ctypes.c_int32), ("bits_per_normal", ctypes.c_int32)]
 
 
+class ZgrCoeffDelivery(ctypes.Structure):
+    _fields_ = [("tensor", ctypes.c_int32), ("q", ctypes.c_void_p), ("scale", ctypes.c_void_p), ("zero", ctypes.c_void_p)]
+
+
 class ZgrKernelTime(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int32), ("dtype", ctypes.c_int32), ("kpad", ctypes.c_int32), ("launches", ctypes.c_int32),
                 ("elements", ctypes.c_int64), ("ms_total", ctypes.c_double)]
@@ -76,6 +80,10 @@ def lib() -> ctypes.CDLL:
         L.zgr_adapt_alpha.restype = ctypes.c_int
         L.zgr_build_subspace.argtypes = [vp, i32, vp, i32, vp]
         L.zgr_build_subspace.restype = ctypes.c_int
+        L.zgr_set_coeffs_dtc_rows.argtypes = [vp, i32, vp, vp, vp, i32, i32]
+        L.zgr_set_coeffs_dtc_rows.restype = ctypes.c_int
+        L.zgr_perturb_layers.argtypes = [vp, u64, dbl, i32, ctypes.POINTER(i32), i32, ctypes.POINTER(ZgrCoeffDelivery), vp, vp]
+        L.zgr_perturb_layers.restype = ctypes.c_int
         L.zgr_get_scalars.argtypes = [vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
         L.zgr_get_state.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(u64), ctypes.POINTER(dbl)]
         L.zgr_update_subspace.argtypes = [vp, i32, vp, i32, vp]
@@ -205,6 +213,28 @@ class Zgr:
         self._keep.append((q, scale, zero))
         _check(lib().zgr_set_coeffs_dtc(self._h, tensor, q.data_ptr(), scale.data_ptr(), None if zero is None else zero.data_ptr(), bits),
                "zgr_set_coeffs_dtc")
+
+    def set_coeffs_dtc_rows(self, tensor: int, q, scale, zero, bits: int, n_rows: int) -> None:
+        """Only the first n_rows rows of the tensor's coefficients come from codes (zgr_set_coeffs_dtc_rows)."""
+        self._keep.append((q, scale, zero))
+        _check(lib().zgr_set_coeffs_dtc_rows(self._h, tensor, q.data_ptr(), scale.data_ptr(), None if zero is None else zero.data_ptr(), bits, n_rows),
+               "zgr_set_coeffs_dtc_rows")
+
+    def perturb_layers(self, seed: int, scale: float, layer_end: Sequence[int], deliveries=(), stream=None, copy_stream=None) -> None:
+        """Layer-wise perturbation with the compressed coefficients of each layer arriving from the host on
+        `copy_stream` while earlier layers are swept (zgr_perturb_layers).  deliveries: tuples
+        (tensor, q_host, scale_host, zero_host or None) of host tensors (pinned for overlap)."""
+        nl, nd = len(layer_end), len(deliveries)
+        arr = (ZgrCoeffDelivery * max(nd, 1))()
+        for i, (l, q, sc, ze) in enumerate(deliveries):
+            assert not q.is_cuda and not sc.is_cuda and q.is_contiguous() and sc.is_contiguous()
+            arr[i] = ZgrCoeffDelivery(l, q.data_ptr(), sc.data_ptr(), None if ze is None else ze.data_ptr())
+        self._keep.append(list(deliveries))
+        if copy_stream is None:
+            import torch
+            copy_stream = torch.cuda.current_stream()
+        _check(lib().zgr_perturb_layers(self._h, seed, scale, nl, (ctypes.c_int32 * nl)(*layer_end), nd, arr, _stream_ptr(stream),
+                                        ctypes.c_void_p(copy_stream.cuda_stream)), "zgr_perturb_layers")
 
     def clear_coeffs(self, tensor: int) -> None:
         _check(lib().zgr_clear_coeffs(self._h, tensor), "zgr_clear_coeffs")

@@ -118,14 +118,22 @@ class Pair:
         self.a, self.b = oracle.mix_scalars(alpha, self.d, self.K, scale_mode)
         self.theta_max = max(float(t.abs().max()) for t in self.theta)
 
-    def set_dtc(self, l: int, q: np.ndarray, scale: np.ndarray, zero=None, bits: int = 8):
+    def set_dtc(self, l: int, q: np.ndarray, scale: np.ndarray, zero=None, bits: int = 8, n_rows=None):
         """q: rank x cols codes (int8 for bits = 8, unsigned values 0..15 for bits = 4).  The oracle keeps the
-        codes as given; for bits = 4 the library receives them packed two to a byte (oracle.dtc_pack4)."""
-        self.q[l] = torch.from_numpy(q).to(self.device)
-        self.scale[l] = torch.from_numpy(scale).to(self.device)
-        self.zero[l] = None if zero is None else torch.from_numpy(zero).to(self.device)
+        codes as given; for bits = 4 the library receives them packed two to a byte (oracle.dtc_pack4).
+        n_rows: only the first n_rows rows are delivered as codes (the others are drawn from the seed)."""
+        if n_rows is not None:
+            q, scale, zero = q[:n_rows], scale[:n_rows], None if zero is None else zero[:n_rows]
+        self.q[l] = torch.from_numpy(np.ascontiguousarray(q)).to(self.device)
+        self.scale[l] = torch.from_numpy(np.ascontiguousarray(scale)).to(self.device)
+        self.zero[l] = None if zero is None else torch.from_numpy(np.ascontiguousarray(zero)).to(self.device)
         payload = self.q[l] if bits == 8 else torch.from_numpy(oracle.dtc_pack4(q)).to(self.device)
-        self.lib.set_coeffs_dtc(l, payload, self.scale[l], self.zero[l], bits)
+        self.payload = getattr(self, "payload", {})
+        self.payload[l] = payload
+        if n_rows is None:
+            self.lib.set_coeffs_dtc(l, payload, self.scale[l], self.zero[l], bits)
+        else:
+            self.lib.set_coeffs_dtc_rows(l, payload, self.scale[l], self.zero[l], bits, n_rows)
 
     def oracle_tensor(self, l: int) -> oracle.OracleTensor:
         (m, n) = self.shapes[l]
