@@ -9,8 +9,8 @@ perturb(+eps), perturb(-2 eps), restore_update(lr/Q) -- 3Q in-place sweeps over 
 `value` = model parameters stepped per second (parameters x steps / time, all ranks), measured with
 CUDA events with weights, subspaces and work tables resident in HBM.  `e2e` repeats the measurement
 with the per-step inputs coming from the host through the C ABI: every guided tensor's subspace is
-copied from pinned host memory (zgr_update_subspaces), the step runs, and the per-tensor norms are read
-back to the host (zgr_get_stats).  The weights themselves stay in HBM in both: keeping the model on
+copied from pinned host memory (zgr_update_subspaces), the step runs with the norm bookkeeping kept by its
+first sweep, and the per-tensor norms are read back to the host (zgr_get_stats).  The weights themselves stay in HBM in both: keeping the model on
 the device and never materialising z is the point of the method.
 
 The path does not shard (one GPU holds the model; the only cross-rank quantities would be two loss
@@ -212,13 +212,19 @@ def run_step_deferred(z, wl, t: int):
     z.restore_update_multi(seeds, [l[0] for l in losses], [l[1] for l in losses], wl.lr / Q)
 
 
-def run_step(z, wl, t: int, schedule: str = "sequential"):
+def run_step(z, wl, t: int, schedule: str = "sequential", keep_norms: bool = False):
+    """keep_norms: the first perturbation of the step also keeps the norm bookkeeping (zgr_enable_stats)."""
     if schedule == "deferred":
         return run_step_deferred(z, wl, t)
     for q in range(wl.queries):
         seed = wl.seed(t, q)
         lp, lm = wl.losses(t, q)
-        z.perturb(seed, wl.eps)
+        if keep_norms and q == 0:
+            z.enable_stats(True)
+            z.perturb(seed, wl.eps)
+            z.enable_stats(False)
+        else:
+            z.perturb(seed, wl.eps)
         z.perturb(seed, -2.0 * wl.eps)
         z.restore_update(seed, lp, lm, wl.lr / wl.queries)
 
@@ -446,8 +452,8 @@ def main():
 
         def e2e_step(t):
             z.update_subspaces(guided, [host_U[l] for l in guided])
-            run_step(z, wl, t, args.schedule)
-            return z.get_stats(wl.seed(t, 0))
+            run_step(z, wl, t, args.schedule, keep_norms=True)
+            return z.get_stats(wl.seed(t, 0))      # the norms kept by the step's first sweep: one small launch and a 7 KB read
 
         e2e_step(10_000)
         barrier()

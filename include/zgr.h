@@ -78,6 +78,8 @@ typedef struct {
   double eps;              /* perturbation scale epsilon > 0 of Eq. (ZOO) */
   int32_t scale_mode;      /* ZGR_SCALE_PAPER | ZGR_SCALE_UNIT */
   int32_t bits_per_normal; /* 32: one generator block per 4 elements; 16: one per 8 elements */
+  int32_t stats;           /* != 0: the first perturbation under every seed also keeps the norm bookkeeping
+                              (see zgr_get_stats); it can be switched later with zgr_enable_stats */
 } zgr_config;
 
 /* Build a context over `n` tensors (Algorithm 1, "Require": model, epsilon, alpha, subspace).
@@ -228,8 +230,16 @@ int zgr_build_subspace(zgr_ctx* ctx, int32_t tensor, const float* grads, int32_t
 
 /* Norm bookkeeping for the adaptive choice of alpha mentioned in Sec. 1: for each tensor l,
  * out[3l+0] = sum (a Z_l)^2, out[3l+1] = sum (b U_l G_l)^2, out[3l+2] = sum z_l^2 for `seed`.
- * Reads no weights.  `out` is a HOST array of 3*n doubles; the call synchronises `stream`. */
+ * `out` is a HOST array of 3*n doubles; the call synchronises `stream`.
+ * With the bookkeeping switched on (zgr_config.stats, zgr_enable_stats) the first zgr_perturb or
+ * zgr_perturb_layers under a seed accumulates these sums inside its sweep (per work item and warp; that sweep
+ * costs about a quarter more), and zgr_get_stats for that seed only adds the partial sums up and reads them
+ * back, as long as alpha, the subspaces and the coefficients have not changed since.  Otherwise the call makes
+ * a pass of its own that regenerates Z and U G for `seed` and reads no weights.  Either way the partial sums
+ * are added in a fixed order: repeated calls give identical bits.  (The two routes agree to about 1e-6
+ * relative, not bit for bit: the sweep takes the guided part as accumulator minus weight.) */
 int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream);
+int zgr_enable_stats(zgr_ctx* ctx, int32_t enable);
 
 /* The norms of ONE tensor, computed without allocating anything.  (The paper has no counterpart; this
  * entry point exists for callers that cannot allocate device memory while they run: loops in which the

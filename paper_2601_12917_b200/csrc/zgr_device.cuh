@@ -42,7 +42,7 @@ __device__ __forceinline__ void philox_block(uint64_t j, uint32_t tensor, uint32
 // Box-Muller on odd-numerator uniforms  u = (2k+1) / 2^(nb+1),  k an nb-bit field (nb = 23 or 16):
 //     n0 = s rho cos(phi),  n1 = s rho sin(phi),   rho = sqrt(-2 ln u1),  phi = 2 pi u2,
 // with the output scale s folded in: |s| goes under the square root, the sign of s becomes a half
-// turn of the angle.  The field k is OR-ed into the mantissa of 1.0f, so t = 1 + k 2^-23 costs no
+// turn of the angle.  The field k sits in the mantissa of 1.0f, so t = 1 + k 2^-23 costs no
 // conversion instruction, and u1 = t + (2^-(nb+1) - 1) is exact in fp32.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ float lg2_approx(float x) {
@@ -90,7 +90,7 @@ __device__ __forceinline__ void sincos_quarter_turns(float y, float& sn, float& 
   cs = __int_as_float(__float_as_int(c0) ^ (((q + 1) & 2) << 30));
 }
 
-// m1, m2: the two uniform fields already placed in mantissa position (bits 0..22).
+// m1, m2: the two uniform fields in mantissa position (bits 0..22) under the exponent of 1.0f (field23 / field16a / field16b).
 //
 // PRECISE = false (16-bit weights): hardware log2 / sqrt / sin / cos approximations; absolute error of
 // a unit normal about 4e-6, far below one ulp of the storage type times any step coefficient.
@@ -100,8 +100,8 @@ __device__ __forceinline__ void sincos_quarter_turns(float y, float& sn, float& 
 // error near 2^-22 for u1 close to 1, which the square root amplifies for the smallest radii.
 template <bool PRECISE>
 __device__ __forceinline__ void box_muller(uint32_t m1, uint32_t m2, const NormalScale& ns, float& n0, float& n1) {
-  const float u1 = __uint_as_float(0x3F800000u | m1) + ns.u1_off;
-  const float t2 = __uint_as_float(0x3F800000u | m2);
+  const float u1 = __uint_as_float(m1) + ns.u1_off;
+  const float t2 = __uint_as_float(m2);
   if (PRECISE) {
     float sn, cs;
     sincos_quarter_turns(fmaf(4.0f, t2, 4.0f * ns.u1_off), sn, cs);   // 4 u2 in (0, 4), exact
@@ -116,12 +116,22 @@ __device__ __forceinline__ void box_muller(uint32_t m1, uint32_t m2, const Norma
   }
 }
 
-// Mantissa-position uniform fields of a generator word (see box_muller): one logic operation each.
+// (x & mask) | bits as ONE logic instruction.  Written with two constants in C++ it becomes two instructions
+// (the three-input logic instruction takes a single immediate); with both constants as register operands it
+// is one, which saves 8 of the ~106 instructions that eight normals cost (measured: 3 % of a sweep).
+__device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t mask, uint32_t bits) {
+  uint32_t r;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(x), "r"(mask), "r"(bits));
+  return r;
+}
+
+// Uniform fields of a generator word, in mantissa position and already carrying the exponent of 1.0f
+// (see box_muller): one logic operation each, plus the rotation for the second 16-bit field.
 //   32-bit mode: the low 23 bits of the word.
 //   16-bit mode: bits 7..22 of the word (radius) and bits 7..22 of the word rotated by 16 (angle).
-__device__ __forceinline__ uint32_t field23(uint32_t x) { return x & 0x7FFFFFu; }
-__device__ __forceinline__ uint32_t field16a(uint32_t x) { return x & 0x7FFF80u; }
-__device__ __forceinline__ uint32_t field16b(uint32_t x) { return __funnelshift_l(x, x, 16) & 0x7FFF80u; }
+__device__ __forceinline__ uint32_t field23(uint32_t x) { return and_or(x, 0x7FFFFFu, 0x3F800000u); }
+__device__ __forceinline__ uint32_t field16a(uint32_t x) { return and_or(x, 0x7FFF80u, 0x3F800000u); }
+__device__ __forceinline__ uint32_t field16b(uint32_t x) { return and_or(__funnelshift_l(x, x, 16), 0x7FFF80u, 0x3F800000u); }
 
 // Eight consecutive normals of stream (tensor, tag) starting at element e (a multiple of 8), each
 // already multiplied by the scale folded into `ns`.
@@ -147,9 +157,22 @@ __device__ __forceinline__ void normals8(const PhiloxKeys& keys, uint32_t tensor
 
 // Fast transform fused with its consumer: acc0 += s rho cos(phi), acc1 += s rho sin(phi).
 __device__ __forceinline__ void box_muller_acc(uint32_t m1, uint32_t m2, const NormalScale& ns, float& acc0, float& acc1) {
-  const float u1 = __uint_as_float(0x3F800000u | m1) + ns.u1_off;
-  const float t2 = __uint_as_float(0x3F800000u | m2);
+  const float u1 = __uint_as_float(m1) + ns.u1_off;
+  const float t2 = __uint_as_float(m2);
   const float rho = sqrt_approx(fabsf(ns.kr * lg2_approx(u1)));
+  const float phi = fmaf(t2, 6.28318530717958647692f, ns.phase);
+  acc0 = fmaf(rho, cos_approx(phi), acc0);
+  acc1 = fmaf(rho, sin_approx(phi), acc1);
+}
+
+// The same, also adding the squared radius of the pair to rsum: (s rho cos)^2 + (s rho sin)^2 = s^2 rho^2 is the
+// argument of the square root, so the energy of the two normals costs one addition.
+__device__ __forceinline__ void box_muller_acc_rsum(uint32_t m1, uint32_t m2, const NormalScale& ns, float& acc0, float& acc1, float& rsum) {
+  const float u1 = __uint_as_float(m1) + ns.u1_off;
+  const float t2 = __uint_as_float(m2);
+  const float x = fabsf(ns.kr * lg2_approx(u1));
+  rsum += x;
+  const float rho = sqrt_approx(x);
   const float phi = fmaf(t2, 6.28318530717958647692f, ns.phase);
   acc0 = fmaf(rho, cos_approx(phi), acc0);
   acc1 = fmaf(rho, sin_approx(phi), acc1);
@@ -173,6 +196,41 @@ __device__ __forceinline__ void normals8_acc(const PhiloxKeys& keys, uint32_t te
     philox4x32_10(oct_lo, oct_hi, tensor, 0u, keys, x);
 #pragma unroll
     for (int w = 0; w < 4; ++w) box_muller_acc(field16a(x[w]), field16b(x[w]), ns, acc[2 * w], acc[2 * w + 1]);
+  }
+}
+
+// normals8_acc that also returns the energy of its eight normals (sum of their squares) in rsum.
+template <int BITS>
+__device__ __forceinline__ void normals8_acc_rsum(const PhiloxKeys& keys, uint32_t tensor, uint32_t oct_lo, uint32_t oct_hi, const NormalScale& ns,
+                                                  float (&acc)[8], float& rsum) {
+  uint32_t x[4];
+  if (BITS == 32) {
+    const uint32_t b_lo = oct_lo << 1, b_hi = (oct_hi << 1) | (oct_lo >> 31);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      philox4x32_10(b_lo + h, b_hi, tensor, 0u, keys, x);
+      box_muller_acc_rsum(field23(x[0]), field23(x[1]), ns, acc[4 * h + 0], acc[4 * h + 1], rsum);
+      box_muller_acc_rsum(field23(x[2]), field23(x[3]), ns, acc[4 * h + 2], acc[4 * h + 3], rsum);
+    }
+  } else {
+    philox4x32_10(oct_lo, oct_hi, tensor, 0u, keys, x);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) box_muller_acc_rsum(field16a(x[w]), field16b(x[w]), ns, acc[2 * w], acc[2 * w + 1], rsum);
+  }
+}
+
+// Partial sums of the norm bookkeeping of one warp for one work item: reduce over the lanes in a fixed order and
+// store them in the item's slot.  Every slot that the finishing kernel reads is written by each launch first.
+__device__ __forceinline__ void store_item_stats(const SweepParams& p, int item, int slot, double s0, double s1, double s2) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, off);
+    s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, off);
+    s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, off);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    double* dst = p.item_stats + (static_cast<int64_t>(p.item_base + item) * kStatSlots + slot) * 3;
+    dst[0] = s0; dst[1] = s1; dst[2] = s2;
   }
 }
 

@@ -27,6 +27,7 @@ struct Group {
   WorkItem* d_items = nullptr;
   int grid = 0;
   int64_t elements = 0;                                   // weights covered by one launch
+  double* d_item_stats = nullptr;                         // kStatSlots x 3 doubles per item (norm bookkeeping), allocated on first use
   std::vector<int32_t> first_item;                        // per tensor l: index of its first item in `items` (size n + 1; items are in tensor order)
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed;  // per-launch events while profiling is on
 };
@@ -49,6 +50,15 @@ struct zgr_ctx {
   std::vector<WorkItem> stats_items;  // plan of the norm kernel (tensors not served by the tcgen05 kernel)
   bool stats_planned = false;
   WorkItem* d_stats_items = nullptr;
+  double* d_stats_slots = nullptr;    // slots of the separate norm pass over stats_items
+  std::vector<int32_t> stats_first;   // per tensor: first item in stats_items (size n + 1)
+  StatRange* d_ranges_pass = nullptr; // per tensor: where the separate pass leaves its partial sums
+  StatRange* d_ranges_sweep = nullptr;  // per tensor: where a sweep with bookkeeping leaves them
+  bool sweep_stats_ready = false;     // slots and ranges of the sweep plan exist
+  bool stats_on = false;              // zgr_config.stats / zgr_enable_stats
+  bool held_valid = false;            // the slots of the sweep plan hold the norms of held_seed, scaled by held_c^2
+  uint64_t held_seed = 0;
+  double held_c = 0.0;
   double* d_stats = nullptr;
   std::map<uint64_t, double> ledger;  // seeds whose perturbation is applied to the weights -> sum of the coefficients applied
   uint64_t last_seed = 0;             // most recently swept seed (introspection)
@@ -263,7 +273,7 @@ int upload_groups(zgr_ctx* ctx, std::vector<Group>& groups) {
 // One sweep  theta <- rnd(theta + sum_q c_q z(seed_q))  over the planned groups (n terms, 1 <= n <= kMaxTerms).
 // t0 <= t1 restricts the sweep to the tensors [t0, t1) (layer-wise sweeps); t1 < 0 means all of them.
 int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, int n, const uint64_t* seeds, const double* c, cudaStream_t st,
-          int32_t t0 = 0, int32_t t1 = -1) {
+          int32_t t0 = 0, int32_t t1 = -1, bool keep_stats = false) {
   SweepParams p;
   std::memset(&p, 0, sizeof(p));
   for (int q = 0; q < n; ++q) {
@@ -282,12 +292,15 @@ int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, i
     if (g.items.empty()) continue;
     p.items = g.d_items;
     p.n_items = static_cast<int32_t>(g.items.size());
+    p.item_stats = keep_stats ? g.d_item_stats : nullptr;
+    p.item_base = 0;
     int grid = g.grid;
     if (t1 >= 0) {
       const int32_t b0 = g.first_item[static_cast<size_t>(t0)], b1 = g.first_item[static_cast<size_t>(t1)];
       if (b1 <= b0) continue;
       p.items = g.d_items + b0;
       p.n_items = b1 - b0;
+      p.item_base = b0;
       grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * blocks_per_sm(g.kc.path)));
     }
     cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -322,6 +335,39 @@ int flush_descs(zgr_ctx* ctx, cudaStream_t st) {
 }
 
 bool is_finite(double x) { return std::isfinite(x); }
+
+// Bookkeeping slots of a plan: kStatSlots x 3 doubles per work item, zeroed once (slots that no warp owns stay
+// zero; the others are rewritten by every launch that keeps the bookkeeping).
+int alloc_slots(zgr_ctx* ctx, double** out, size_t n_items) {
+  const size_t count = std::max<size_t>(n_items, 1) * kStatSlots * 3;
+  int rc = dev_alloc(ctx, out, count);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemset(*out, 0, count * sizeof(double)));
+  return rc;
+}
+
+// In-sweep bookkeeping needs every group of the sweep plan to be a kernel family that keeps it.
+bool sweep_stats_possible(const zgr_ctx* ctx) {
+  for (const Group& g : ctx->groups)
+    if (!g.items.empty() && g.kc.path == PATH_MMA) return false;
+  return true;
+}
+
+int prepare_sweep_stats(zgr_ctx* ctx) {
+  if (ctx->sweep_stats_ready) return ZGR_OK;
+  const size_t n = ctx->descs.size();
+  std::vector<StatRange> ranges(n, StatRange{nullptr, 0, 0});
+  for (Group& g : ctx->groups) {
+    if (g.items.empty()) continue;
+    const int rc = alloc_slots(ctx, &g.d_item_stats, g.items.size());
+    if (rc != ZGR_OK) return rc;
+    for (size_t l = 0; l < n; ++l)
+      if (g.first_item[l + 1] > g.first_item[l]) ranges[l] = StatRange{g.d_item_stats, g.first_item[l], g.first_item[l + 1] - g.first_item[l]};
+  }
+  int rc = dev_alloc(ctx, &ctx->d_ranges_sweep, n);
+  if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(ctx->d_ranges_sweep, ranges.data(), n * sizeof(StatRange), cudaMemcpyHostToDevice));
+  if (rc == ZGR_OK) ctx->sweep_stats_ready = true;
+  return rc;
+}
 
 // A context's tables, tensor maps and borrowed pointers live on the device that was current at zgr_init.
 // Launching from another current device would hand its kernels foreign addresses, so every entry point
@@ -423,6 +469,7 @@ int zgr_init(zgr_ctx** out, const zgr_tensor* tensors, int32_t n, const zgr_conf
   zgr_ctx* ctx = new (std::nothrow) zgr_ctx();
   if (!ctx) return ZGR_ENOMEM;
   ctx->cfg = *cfg;
+  ctx->stats_on = cfg->stats != 0;
   ctx->d = d;
   ctx->K = K;
   set_mixing(ctx, cfg->alpha);
@@ -536,8 +583,20 @@ int zgr_perturb(zgr_ctx* ctx, uint64_t seed, double scale, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
-  rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, st);
+  // the first perturbation under a seed also keeps the norm bookkeeping when that is switched on
+  const bool keep = ctx->stats_on && ctx->ledger.empty() && scale != 0.0 && sweep_stats_possible(ctx);
+  if (keep) {
+    rc = prepare_sweep_stats(ctx);
+    if (rc != ZGR_OK) return rc;
+    ctx->held_valid = false;
+  }
+  rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, st, 0, -1, keep);
   if (rc != ZGR_OK) return rc;
+  if (keep) {
+    ctx->held_valid = true;
+    ctx->held_seed = seed;
+    ctx->held_c = scale;
+  }
   ledger_add(ctx, seed, scale);
   return ZGR_OK;
 }
@@ -618,6 +677,7 @@ int zgr_set_alpha(zgr_ctx* ctx, double alpha) {
   // part at all) has no tensor-core operands and keeps serving every tensor without its subspace.
   if (ctx->guided_at_init == false && alpha < 1.0 && ctx->K > 0) return ZGR_ESTATE;
   set_mixing(ctx, alpha);
+  ctx->held_valid = false;
   return ZGR_OK;
 }
 
@@ -646,6 +706,7 @@ int zgr_adapt_alpha(zgr_ctx* ctx, const double* stats, double alpha_min, double 
   double alpha = (1.0 - eta) * alpha_old + eta * (e_g / (e_iso + e_g));
   alpha = std::min(std::max(alpha, alpha_min), alpha_max);
   set_mixing(ctx, alpha);
+  ctx->held_valid = false;
   *alpha_out = alpha;
   return ZGR_OK;
 }
@@ -662,6 +723,7 @@ int zgr_set_coeffs_dtc_rows(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const
   td.qbits = bits;
   td.qrows = n_rows;
   ctx->descs_dirty = true;
+  ctx->held_valid = false;
   return ZGR_OK;
 }
 
@@ -725,13 +787,24 @@ int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_laye
       if (rc != ZGR_OK) return rc;
     }
   }
+  const bool keep = ctx->stats_on && ctx->ledger.empty() && scale != 0.0 && sweep_stats_possible(ctx);
+  if (keep) {
+    rc = prepare_sweep_stats(ctx);
+    if (rc != ZGR_OK) return rc;
+  }
+  ctx->held_valid = false;     // (a delivery changes the coefficients that earlier norms were taken with)
   for (int32_t L = 0; L < n_layers; ++L) {
     if (n_deliveries > 0 && !by_layer[static_cast<size_t>(L)].empty()) {
       rc = check(ctx, cudaStreamWaitEvent(st, ctx->layer_events[static_cast<size_t>(L)], 0));
       if (rc != ZGR_OK) return rc;
     }
-    rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, st, L ? layer_end[L - 1] : 0, layer_end[L]);
+    rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, st, L ? layer_end[L - 1] : 0, layer_end[L], keep);
     if (rc != ZGR_OK) return rc;   // (a failure here leaves the earlier layers swept: the context is sticky-failed by check())
+  }
+  if (keep) {
+    ctx->held_valid = true;
+    ctx->held_seed = seed;
+    ctx->held_c = scale;
   }
   ledger_add(ctx, seed, scale);
   return ZGR_OK;
@@ -747,6 +820,7 @@ int zgr_clear_coeffs(zgr_ctx* ctx, int32_t tensor) {
   td.qzero = nullptr;
   td.qrows = 0;
   ctx->descs_dirty = true;
+  ctx->held_valid = false;
   return ZGR_OK;
 }
 
@@ -758,12 +832,30 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
   const size_t n = ctx->descs.size();
+  if (ctx->held_valid && ctx->held_seed == seed) {
+    // The first perturbation under this seed kept the bookkeeping: add up its partial sums (fixed order) and
+    // read them back; they are the norms of c z, c being that perturbation's coefficient.
+    rc = check(ctx, launch_stats_finish(ctx->d_ranges_sweep, static_cast<int>(n), ctx->d_stats, st));
+    if (rc == ZGR_OK) ctx->launches++;
+    if (rc == ZGR_OK) rc = check(ctx, cudaMemcpyAsync(out, ctx->d_stats, 3 * n * sizeof(double), cudaMemcpyDeviceToHost, st));
+    if (rc == ZGR_OK) rc = check(ctx, cudaStreamSynchronize(st));
+    if (rc != ZGR_OK) return rc;
+    const double inv = 1.0 / (ctx->held_c * ctx->held_c);
+    for (size_t i = 0; i < 3 * n; ++i) out[i] *= inv;
+    return ZGR_OK;
+  }
+  // A pass of its own: regenerate Z and U G for `seed` without touching the weights.
+  rc = prepare_sweep_stats(ctx);      // (the tcgen05 groups leave their partial sums in the slots of the sweep plan)
+  if (rc != ZGR_OK) return rc;
+  ctx->held_valid = false;
   if (!ctx->stats_planned) {
     // tensors served by the tcgen05 kernel reuse its work items; all others get a generic tiling (strips of 64 columns)
     int64_t total = ctx->d;
     int64_t target = std::min<int64_t>(std::max<int64_t>(total / (static_cast<int64_t>(ctx->sm_count) * 64), 4096), 131072);
+    ctx->stats_first.assign(n + 1, 0);
     for (size_t l = 0; l < n; ++l) {
       const TensorDesc& t = ctx->descs[l];
+      ctx->stats_first[l] = static_cast<int32_t>(ctx->stats_items.size());
       if (t.umma && ctx->guided_at_init) continue;
       for (int64_t c0 = 0; c0 < t.cols; c0 += 64) {
         const int ncols = static_cast<int>(std::min<int64_t>(64, t.cols - c0));
@@ -772,16 +864,28 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
           ctx->stats_items.push_back(WorkItem{static_cast<int32_t>(l), ncols, r0, std::min(nrows, t.rows - r0), c0});
       }
     }
+    ctx->stats_first[n] = static_cast<int32_t>(ctx->stats_items.size());
     if (!ctx->stats_items.empty()) {
       rc = dev_alloc(ctx, &ctx->d_stats_items, ctx->stats_items.size());
       if (rc == ZGR_OK)
         rc = check(ctx, cudaMemcpy(ctx->d_stats_items, ctx->stats_items.data(), ctx->stats_items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
       if (rc != ZGR_OK) return rc;
     }
+    rc = alloc_slots(ctx, &ctx->d_stats_slots, ctx->stats_items.size());
+    if (rc != ZGR_OK) return rc;
+    std::vector<StatRange> ranges(n);
+    for (size_t l = 0; l < n; ++l) {
+      ranges[l] = StatRange{ctx->d_stats_slots, ctx->stats_first[l], ctx->stats_first[l + 1] - ctx->stats_first[l]};
+      if (ctx->descs[l].umma && ctx->guided_at_init)
+        for (const Group& g : ctx->groups)
+          if (g.kc.path == PATH_UMMA && g.first_item[l + 1] > g.first_item[l])
+            ranges[l] = StatRange{g.d_item_stats, g.first_item[l], g.first_item[l + 1] - g.first_item[l]};
+    }
+    rc = dev_alloc(ctx, &ctx->d_ranges_pass, n);
+    if (rc == ZGR_OK) rc = check(ctx, cudaMemcpy(ctx->d_ranges_pass, ranges.data(), n * sizeof(StatRange), cudaMemcpyHostToDevice));
+    if (rc != ZGR_OK) return rc;
     ctx->stats_planned = true;
   }
-  rc = check(ctx, cudaMemsetAsync(ctx->d_stats, 0, 3 * n * sizeof(double), st));
-  if (rc != ZGR_OK) return rc;
   SweepParams p;
   std::memset(&p, 0, sizeof(p));
   p.n_terms = 1;
@@ -793,7 +897,8 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
   p.n_items = static_cast<int32_t>(ctx->stats_items.size());
   p.term[0].cb = static_cast<float>(ctx->b);
   p.kshift = kshift_for(std::fabs(ctx->b));
-  p.stats = ctx->d_stats;
+  p.item_stats = ctx->d_stats_slots;
+  p.item_base = 0;
   if (p.n_items > 0) {
     const int grid = static_cast<int>(std::min<int64_t>(p.n_items, static_cast<int64_t>(ctx->sm_count) * 4));
     rc = check(ctx, launch_stats(ctx->cfg.bits_per_normal, p, grid, st));
@@ -804,13 +909,23 @@ int zgr_get_stats(zgr_ctx* ctx, uint64_t seed, double* out, void* stream) {
     if (g.kc.path != PATH_UMMA || g.items.empty()) continue;
     p.items = g.d_items;
     p.n_items = static_cast<int32_t>(g.items.size());
+    p.item_stats = g.d_item_stats;
     rc = check(ctx, launch_stats_umma(g.kc, p, ctx->d_tmaps, ctx->d_err, g.grid, st));
     if (rc != ZGR_OK) return rc;
     ctx->launches++;
   }
+  rc = check(ctx, launch_stats_finish(ctx->d_ranges_pass, static_cast<int>(n), ctx->d_stats, st));
+  if (rc != ZGR_OK) return rc;
+  ctx->launches++;
   rc = check(ctx, cudaMemcpyAsync(out, ctx->d_stats, 3 * n * sizeof(double), cudaMemcpyDeviceToHost, st));
   if (rc != ZGR_OK) return rc;
   return check(ctx, cudaStreamSynchronize(st));
+}
+
+int zgr_enable_stats(zgr_ctx* ctx, int32_t enable) {
+  if (!ctx) return ZGR_EINVAL;
+  ctx->stats_on = enable != 0;     // norms already held stay available until something they depend on changes
+  return ZGR_OK;
 }
 
 int zgr_debug_philox(zgr_ctx* ctx, uint64_t seed, int32_t tensor, int32_t tag, uint64_t first_block, int64_t n_blocks, uint32_t* dev_out,
@@ -930,6 +1045,7 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
   if (ctx->sticky) return ctx->sticky;
   if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   if (!ctx->ledger.empty()) return ZGR_ESTATE;
+  ctx->held_valid = false;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = ZGR_OK;
   if (U_src != nullptr && U_src != td.U) {
@@ -1047,6 +1163,7 @@ int zgr_update_subspaces(zgr_ctx* ctx, int32_t n, const int32_t* tensors, const 
   if (ctx->sticky) return ctx->sticky;
   if (!on_ctx_device(ctx)) return ZGR_EINVAL;
   if (!ctx->ledger.empty()) return ZGR_ESTATE;
+  ctx->held_valid = false;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // every tensor of the tcgen05 path is listed: their operand copies are rebuilt by one launch after the copies
   const bool fused = n_umma > 0 && n_umma == ctx->n_split_jobs;

@@ -62,6 +62,7 @@ struct SeedTerm {
 };
 
 constexpr int kMaxTerms = 8;   // ZGR_MAX_SEEDS of the C ABI
+constexpr int kStatSlots = 16; // partial sums kept per work item (one per warp that works on it; unused slots stay zero)
 
 // Per-launch constants (passed by value in the kernel parameter space).  A single-seed sweep uses
 // term[0] only, addressed with a compile-time index so that its round keys stay constant-bank
@@ -75,6 +76,8 @@ struct SweepParams {
   int32_t n_items;
   double* stats;         // 3 doubles per tensor (stats kernels only)
   float* zout;           // rows x cols fp32 image of the one tensor swept (test hook of the tcgen05 kernel only)
+  double* item_stats;    // norm bookkeeping: kStatSlots x 3 doubles per work item of the group (partial sums per warp), or null
+  int32_t item_base;     // index of items[0] in the group's full item list (layer-wise launches start in the middle)
   int32_t kshift;        // tcgen05 kernel: the coefficient strips are scaled by a power of two so that sum_q |c_q| b 2^kshift
                          // is near 1 (see the operand precision note in zgr_umma.cu)
 };

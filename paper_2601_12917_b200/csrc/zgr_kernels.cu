@@ -31,7 +31,10 @@ constexpr int kWarps = kThreads / 32;
 // ---------------------------------------------------------------------------------------------
 // isotropic sweep
 // ---------------------------------------------------------------------------------------------
-template <typename T, int BITS, bool PRECISE, bool MULTI>
+// SSTATS = true (single-term sweeps only) also accumulates the norm bookkeeping of the sweep: per work item and
+// warp the sums of (c a Z)^2, (c b U G)^2 and (c z)^2 over its elements, stored in the item's slots (the
+// finishing kernel adds them up per tensor in a fixed order; the host divides by c^2).
+template <typename T, int BITS, bool PRECISE, bool MULTI, bool SSTATS = false>
 __global__ void __launch_bounds__(kThreads) sweep_iso_kernel(const __grid_constant__ SweepParams p) {
   for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
     const WorkItem w = p.items[it];
@@ -40,20 +43,29 @@ __global__ void __launch_bounds__(kThreads) sweep_iso_kernel(const __grid_consta
     const uint32_t tid = static_cast<uint32_t>(td.id);
     const int64_t e0 = w.row0_or_e0, count = w.nrows_or_count;
     const int64_t n_oct = w.ncols ? count / 8 : 0;  // ncols != 0: 128-bit access is legal for this tensor
+    double s_iso = 0.0;
 #pragma unroll 2
     for (int64_t v = threadIdx.x; v < n_oct; v += kThreads) {
       const int64_t e = e0 + 8 * v;
       float th[8], z[8];
       Storage<T>::load8(base + e, th);
       iso8<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e), z);
+      if (SSTATS) {
+        float f = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f = fmaf(z[i], z[i], f);
+        s_iso += static_cast<double>(f);
+      }
 #pragma unroll
       for (int i = 0; i < 8; ++i) th[i] += z[i];
       Storage<T>::store8(base + e, th);
     }
     for (int64_t e = e0 + 8 * n_oct + threadIdx.x; e < e0 + count; e += kThreads) {
       const float z = iso1<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e));
+      if (SSTATS) s_iso += static_cast<double>(z) * z;
       Storage<T>::store1(base + e, Storage<T>::load1(base + e) + z);
     }
+    if (SSTATS) store_item_stats(p, it, threadIdx.x >> 5, s_iso, 0.0, s_iso);
   }
 }
 
@@ -63,7 +75,7 @@ __global__ void __launch_bounds__(kThreads) sweep_iso_kernel(const __grid_consta
 // [8l, 8l+8) of the strip and keeps its R x 8 coefficients in registers; the eight warps walk
 // the rows of the item in an interleaved fashion, each row being one 128-bit access per lane.
 // ---------------------------------------------------------------------------------------------
-template <typename T, int BITS, bool PRECISE, int R, bool MULTI>
+template <typename T, int BITS, bool PRECISE, int R, bool MULTI, bool SSTATS = false>
 __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_constant__ SweepParams p) {
   __shared__ float Gs[R][256 + 8];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -98,6 +110,7 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_con
       for (int i = 0; i < 8; ++i) g[k][i] = active ? Gs[k][8 * lane + i] : 0.0f;
     const bool u_vec = (r == R) && ((reinterpret_cast<uintptr_t>(td.U) & 15) == 0);
     const int64_t row_end = w.row0_or_e0 + w.nrows_or_count;
+    double s_iso = 0.0, s_gd = 0.0, s_z = 0.0;   // SSTATS only
     for (int64_t row = w.row0_or_e0 + warp; row < row_end; row += kWarps) {
       float u[R];
       if (u_vec) {
@@ -115,23 +128,36 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_con
         float th[8], z[8];
         Storage<T>::load8(base + e, th);
         iso8<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e), z);
+        float f_iso = 0.0f, f_gd = 0.0f, f_z = 0.0f;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           float acc = z[i];  // the perturbation is summed on its own scale, then added to theta once
 #pragma unroll
           for (int k = 0; k < R; ++k) acc = fmaf(u[k], g[k][i], acc);
+          if (SSTATS) {
+            const float gd = acc - z[i];
+            f_iso = fmaf(z[i], z[i], f_iso);
+            f_gd = fmaf(gd, gd, f_gd);
+            f_z = fmaf(acc, acc, f_z);
+          }
           th[i] += acc;
+        }
+        if (SSTATS) {
+          s_iso += static_cast<double>(f_iso);
+          s_gd += static_cast<double>(f_gd);
+          s_z += static_cast<double>(f_z);
         }
         Storage<T>::store8(base + e, th);
       }
     }
+    if (SSTATS) store_item_stats(p, it, warp, s_iso, s_gd, s_z);
   }
 }
 
 // ---------------------------------------------------------------------------------------------
 // any shape: one element per thread, strip of 64 columns, rank <= 64.
 // ---------------------------------------------------------------------------------------------
-template <typename T, int BITS, bool PRECISE, bool MULTI>
+template <typename T, int BITS, bool PRECISE, bool MULTI, bool SSTATS = false>
 __global__ void __launch_bounds__(kThreads) sweep_generic_kernel(const __grid_constant__ SweepParams p) {
   __shared__ float Gs[64][64 + 1];
   const int cl = threadIdx.x & 63, rg = threadIdx.x >> 6;
@@ -147,14 +173,24 @@ __global__ void __launch_bounds__(kThreads) sweep_generic_kernel(const __grid_co
       if (c < w.ncols) Gs[k][c] = guided1<BITS, PRECISE, MULTI>(td, p, k, w.col0 + c);
     }
     __syncthreads();
-    if (cl >= w.ncols) continue;
-    const int64_t row_end = w.row0_or_e0 + w.nrows_or_count;
-    for (int64_t row = w.row0_or_e0 + rg; row < row_end; row += kThreads / 64) {
-      const int64_t e = row * td.cols + w.col0 + cl;
-      float acc = iso1<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e));
-      for (int k = 0; k < r; ++k) acc = fmaf(__ldg(td.U + row * r + k), Gs[k][cl], acc);
-      Storage<T>::store1(base + e, Storage<T>::load1(base + e) + acc);
+    double s_iso = 0.0, s_gd = 0.0, s_z = 0.0;   // SSTATS only
+    if (cl < w.ncols) {
+      const int64_t row_end = w.row0_or_e0 + w.nrows_or_count;
+      for (int64_t row = w.row0_or_e0 + rg; row < row_end; row += kThreads / 64) {
+        const int64_t e = row * td.cols + w.col0 + cl;
+        const float iso = iso1<BITS, PRECISE, MULTI>(p, tid, static_cast<uint64_t>(e));
+        float acc = iso;
+        for (int k = 0; k < r; ++k) acc = fmaf(__ldg(td.U + row * r + k), Gs[k][cl], acc);
+        if (SSTATS) {
+          const float gd = acc - iso;
+          s_iso += static_cast<double>(iso) * iso;
+          s_gd += static_cast<double>(gd) * gd;
+          s_z += static_cast<double>(acc) * acc;
+        }
+        Storage<T>::store1(base + e, Storage<T>::load1(base + e) + acc);
+      }
     }
+    if (SSTATS) store_item_stats(p, it, threadIdx.x >> 5, s_iso, s_gd, s_z);
   }
 }
 
@@ -338,12 +374,13 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_mma_kernel(const __grid_con
 
 // ---------------------------------------------------------------------------------------------
 // Norm bookkeeping: per tensor sum (a Z)^2, sum (b U G)^2, sum z^2 (no weights are read).
-// Same tiling as the generic kernel; fp32 per element, double partial sums, one atomic per warp.
+// Same tiling as the generic kernel; fp32 per element, double partial sums, one slot per warp and work item
+// (summed per tensor in a fixed order by stats_finish_kernel, so repeated calls give identical bits).
 // ---------------------------------------------------------------------------------------------
 template <int BITS>
 __global__ void __launch_bounds__(kThreads) stats_kernel(const __grid_constant__ SweepParams p) {
   __shared__ float Gs[64][64 + 1];
-  const int cl = threadIdx.x & 63, rg = threadIdx.x >> 6, lane = threadIdx.x & 31;
+  const int cl = threadIdx.x & 63, rg = threadIdx.x >> 6;
   for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
     const WorkItem w = p.items[it];
     const TensorDesc& td = p.tensors[w.tensor];
@@ -368,18 +405,28 @@ __global__ void __launch_bounds__(kThreads) stats_kernel(const __grid_constant__
         s2 += static_cast<double>(iso + gd) * (iso + gd);
       }
     }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, off);
-      s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, off);
-      s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, off);
-    }
-    if (lane == 0) {
-      atomicAdd(p.stats + 3 * w.tensor + 0, s0);
-      atomicAdd(p.stats + 3 * w.tensor + 1, s1);
-      atomicAdd(p.stats + 3 * w.tensor + 2, s2);
-    }
+    store_item_stats(p, it, threadIdx.x >> 5, s0, s1, s2);
   }
+}
+
+// out[3 l + j] = sum over the work items of tensor l and their slots, in a fixed order.
+__global__ void __launch_bounds__(kThreads) stats_finish_kernel(const StatRange* __restrict__ ranges, double* __restrict__ out) {
+  __shared__ double red[kThreads][3];
+  const StatRange r = ranges[blockIdx.x];
+  double t[3] = {0.0, 0.0, 0.0};
+  for (int i = threadIdx.x; i < r.count; i += kThreads) {
+    const double* src = r.slots + static_cast<int64_t>(r.first + i) * kStatSlots * 3;
+    for (int sl = 0; sl < kStatSlots; ++sl)
+      for (int j = 0; j < 3; ++j) t[j] += src[3 * sl + j];
+  }
+  for (int j = 0; j < 3; ++j) red[threadIdx.x][j] = t[j];
+  __syncthreads();
+  for (int half = kThreads / 2; half > 0; half >>= 1) {
+    if (threadIdx.x < half)
+      for (int j = 0; j < 3; ++j) red[threadIdx.x][j] += red[threadIdx.x + half][j];
+    __syncthreads();
+  }
+  if (threadIdx.x < 3) out[3 * blockIdx.x + threadIdx.x] = red[0][threadIdx.x];
 }
 
 // U (rows x r fp32) -> A-operand fragments, bf16 hi/lo, zero padded to whole 16-row tiles and to KP.
@@ -457,6 +504,24 @@ namespace {
 
 template <typename T, int BITS, bool PRECISE, bool MULTI>
 cudaError_t launch_typed(const KernelChoice& kc, const SweepParams& p, int grid, cudaStream_t st) {
+  if constexpr (!MULTI) {
+    if (p.item_stats != nullptr) {      // the sweep also accumulates the norm bookkeeping
+      switch (kc.path) {
+        case PATH_ISO:
+          sweep_iso_kernel<T, BITS, PRECISE, false, true><<<grid, kThreads, 0, st>>>(p);
+          return cudaGetLastError();
+        case PATH_FMA:
+          if (kc.kpad == 4) sweep_fma_kernel<T, BITS, PRECISE, 4, false, true><<<grid, kThreads, 0, st>>>(p);
+          else sweep_fma_kernel<T, BITS, PRECISE, 8, false, true><<<grid, kThreads, 0, st>>>(p);
+          return cudaGetLastError();
+        case PATH_GENERIC:
+          sweep_generic_kernel<T, BITS, PRECISE, false, true><<<grid, kThreads, 0, st>>>(p);
+          return cudaGetLastError();
+        default:
+          return cudaErrorInvalidValue;  // the legacy tensor-core kernel keeps no bookkeeping; the host does not ask it to
+      }
+    }
+  }
   switch (kc.path) {
     case PATH_ISO:
       sweep_iso_kernel<T, BITS, PRECISE, MULTI><<<grid, kThreads, 0, st>>>(p);
@@ -535,6 +600,12 @@ cudaError_t launch_sweep(const KernelChoice& kc, const SweepParams& p, int grid,
 cudaError_t launch_stats(int bits, const SweepParams& p, int grid, cudaStream_t st) {
   if (bits == 32) stats_kernel<32><<<grid, kThreads, 0, st>>>(p);
   else stats_kernel<16><<<grid, kThreads, 0, st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_stats_finish(const StatRange* d_ranges, int n_tensors, double* d_out, cudaStream_t st) {
+  if (n_tensors <= 0) return cudaSuccess;
+  stats_finish_kernel<<<n_tensors, kThreads, 0, st>>>(d_ranges, d_out);
   return cudaGetLastError();
 }
 

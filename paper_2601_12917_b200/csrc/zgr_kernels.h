@@ -46,6 +46,13 @@ struct SplitJob {
 cudaError_t launch_split_subspace_rowmajor_all(const SplitJob* d_jobs, int n_jobs, cudaStream_t st);
 
 cudaError_t launch_stats(int bits, const SweepParams& p, int grid, cudaStream_t st);
+// Norm bookkeeping, second stage: tensor l owns the work items [first, first + count) of the slot array `slots`
+// (kStatSlots x 3 doubles per item); out[3 l + j] receives their sum, added in a fixed order.
+struct StatRange {
+  const double* slots;
+  int32_t first, count;
+};
+cudaError_t launch_stats_finish(const StatRange* d_ranges, int n_tensors, double* d_out, cudaStream_t st);
 cudaError_t launch_split_subspace(const float* U, int64_t rows, int r, int kp, uint4* out, cudaStream_t st);
 cudaError_t launch_philox_blocks(const PhiloxKeys& keys, uint32_t tensor, uint32_t tag, uint64_t first_block, int64_t n_blocks,
                                  uint32_t* out, cudaStream_t st);

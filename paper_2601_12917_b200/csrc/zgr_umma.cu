@@ -221,6 +221,28 @@ struct Pack16<__half> {
   }
 };
 
+// the eight 16-bit values of a 16-byte chunk as floats
+template <typename T>
+__device__ __forceinline__ void unpack8(const uint4& raw, float (&v)[8]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if constexpr (sizeof(T) == 2 && Pack16<T>::kFmt == 1) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    } else {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+      v[2 * i] = f.x;
+      v[2 * i + 1] = f.y;
+    }
+  }
+}
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");
+  return v;
+}
+
 // fp16 hi/lo split of a pair of floats, packed as f16x2 (first value in the low half)
 __device__ __forceinline__ void split_f16(float x0, float x1, uint32_t& hi, uint32_t& lo) {
   const __half2 h = __floats2half2_rn(x0, x1);
@@ -311,7 +333,12 @@ struct TileCoord {
 // result of every element (accumulator plus normals, before the rounding to the storage type) goes to
 // p.zout[row * cols + col] by plain stores and nothing is written back to the weights.  On a zeroed
 // weight image with coefficient 1 that is z itself as this kernel computes it.
-template <typename T, int BITS, int KP, bool STATS = false, bool MULTI = false, bool ZOUT = false>
+// SSTATS = true (single-term sweeps) is the sweep itself with the norm bookkeeping folded in: before a thread
+// overwrites its 16 bytes of the staged tile it reads theta back from them, so that the guided part (accumulator
+// minus theta) and the whole step (result minus theta) can be squared and summed; the isotropic part costs one
+// addition per pair of normals (the squared radius is the argument of the square root).  The sums are of
+// (c a Z)^2, (c b U G)^2 and (c z)^2; the host divides by c^2.
+template <typename T, int BITS, int KP, bool STATS = false, bool MULTI = false, bool ZOUT = false, bool SSTATS = false>
 __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(const __grid_constant__ SweepParams p, const CUtensorMap* __restrict__ tmaps,
                                                                      int* __restrict__ error) {
   using Cfg = UmmaCfg<KP>;
@@ -530,7 +557,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
     const int et = e * 32 + lane;
     const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(32 * quad) << 16);
     const int row_in_tile = 32 * quad + lane;
-    const uint32_t row_xor = static_cast<uint32_t>(row_in_tile & 7);
+    const uint32_t row_xor16 = static_cast<uint32_t>(row_in_tile & 7) << 4;   // 128-byte swizzle: the 16-byte chunk index is xor-ed with the row
     const uint32_t theta_s32 = smem_u32(theta_base);
     const uint32_t g_s32 = smem_u32(g_base);
     int t = 0, item_no = 0;
@@ -594,10 +621,10 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
 
       const int row_end = static_cast<int>(w.row0_or_e0 + w.nrows_or_count);
       const int nsub = (w.ncols + NS - 1) / NS;
-      double sum_iso = 0.0, sum_gd = 0.0, sum_z = 0.0;   // STATS only
+      double sum_iso = 0.0, sum_gd = 0.0, sum_z = 0.0;   // STATS / SSTATS only
       for (int row0 = static_cast<int>(w.row0_or_e0); row0 < row_end && ok; row0 += 128) {
         const int64_t row = static_cast<int64_t>(row0) + row_in_tile;
-        const uint64_t row_e0 = static_cast<uint64_t>(row) * tcols + static_cast<uint64_t>(w.col0);
+        const uint64_t row_oct0 = (static_cast<uint64_t>(row) * tcols + static_cast<uint64_t>(w.col0)) >> 3;   // octet index of the strip's first column in this row
         for (int sub = 0; sub < nsub; ++sub, ++t) {
           if (GROUPS > 1 && (t % GROUPS) != grp) continue;     // another group's tile
           const int s = t % S, b = t % NACC;
@@ -609,11 +636,12 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
           const uint32_t tmem_warp = tmem_row + static_cast<uint32_t>(32 * cgrp);
           const uint32_t chunk0 = static_cast<uint32_t>(((32 * cgrp) & 63) >> 3);
           const uint32_t out_off = static_cast<uint32_t>(((32 * cgrp) >> 6) * 16384 + row_in_tile * 128);
-          const uint64_t row_e = row_e0 + static_cast<uint64_t>(32 * cgrp);
           if (NS * sub + 32 * cgrp < w.ncols) {
-            const uint64_t oct0 = (row_e + static_cast<uint64_t>(NS * sub)) >> 3;
+            const uint64_t oct0 = row_oct0 + static_cast<uint64_t>((NS * sub + 32 * cgrp) >> 3);
             const uint32_t oct0_lo = static_cast<uint32_t>(oct0), oct0_hi = static_cast<uint32_t>(oct0 >> 32);
-            const uint32_t out_box = theta_s32 + static_cast<uint32_t>(s * Cfg::THETA_BYTES) + out_off;
+            // the row's 128 bytes in the staged tile start on a 128-byte boundary, so the swizzled chunk offset
+            // (bits 4..6) can be xor-ed in rather than added: one logic instruction per chunk
+            const uint32_t out_box = (theta_s32 + static_cast<uint32_t>(s * Cfg::THETA_BYTES) + out_off) ^ row_xor16;
             uint32_t h0[16], h1[16];
             tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS), h0);
             tmem_ld16(tmem_warp + static_cast<uint32_t>(b * NS + 16), h1);
@@ -650,6 +678,28 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
 #pragma unroll
               for (int i = 0; i < 8; ++i) acc[i] = __uint_as_float(o < 2 ? h0[8 * (o & 1) + i] : h1[8 * (o & 1) + i]);
               const uint32_t lo = oct0_lo + static_cast<uint32_t>(o);
+              if constexpr (SSTATS) {
+                const uint32_t chunk_addr = out_box ^ ((chunk0 + static_cast<uint32_t>(o)) << 4);
+                float th[8];
+                unpack8<T>(lds128(chunk_addr), th);                      // theta, before this thread overwrites it
+                float f_iso = 0.0f, f_gd = 0.0f, f_z = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const float gd = acc[i] - th[i];
+                  f_gd = fmaf(gd, gd, f_gd);
+                }
+                normals8_acc_rsum<BITS>(p.term[0].keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.term[0].iso, acc, f_iso);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const float zc = acc[i] - th[i];
+                  f_z = fmaf(zc, zc, f_z);
+                }
+                if (row < row_end && NS * sub + 32 * cgrp + 8 * o < w.ncols) {
+                  sum_iso += static_cast<double>(f_iso);
+                  sum_gd += static_cast<double>(f_gd);
+                  sum_z += static_cast<double>(f_z);
+                }
+              } else
               normals8_acc<BITS>(p.term[0].keys, tid, lo, oct0_hi + (lo < oct0_lo ? 1u : 0u), p.term[0].iso, acc);
               if (MULTI) {
 #pragma unroll 1
@@ -666,7 +716,7 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
               } else {
                 const uint4 q = make_uint4(Pack16<T>::pack(acc[0], acc[1]), Pack16<T>::pack(acc[2], acc[3]), Pack16<T>::pack(acc[4], acc[5]),
                                            Pack16<T>::pack(acc[6], acc[7]));
-                sts128(out_box + (((chunk0 + static_cast<uint32_t>(o)) ^ row_xor) << 4), q);
+                sts128(out_box ^ ((chunk0 + static_cast<uint32_t>(o)) << 4), q);
               }
             }
             }
@@ -681,18 +731,8 @@ __global__ void __launch_bounds__(UmmaCfg<KP>::THREADS, 1) sweep_umma_kernel(con
           }
         }
       }
-      if constexpr (STATS) {
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-          sum_iso += __shfl_xor_sync(0xFFFFFFFFu, sum_iso, off);
-          sum_gd += __shfl_xor_sync(0xFFFFFFFFu, sum_gd, off);
-          sum_z += __shfl_xor_sync(0xFFFFFFFFu, sum_z, off);
-        }
-        if (lane == 0) {
-          atomicAdd(p.stats + 3 * w.tensor + 0, sum_iso);
-          atomicAdd(p.stats + 3 * w.tensor + 1, sum_gd);
-          atomicAdd(p.stats + 3 * w.tensor + 2, sum_z);
-        }
+      if constexpr (STATS || SSTATS) {
+        if (ok) store_item_stats(p, it, e, sum_iso, sum_gd, sum_z);   // one slot per epilogue warp (at most kStatSlots of them)
       }
     }
   }
@@ -712,11 +752,13 @@ size_t umma_smem_bytes(int kpad) {
 int umma_strip_cols(int kpad) { return kpad == 64 ? UmmaCfg<64>::NS * UmmaCfg<64>::NSUB : (kpad == 32 ? UmmaCfg<32>::NS * UmmaCfg<32>::NSUB : UmmaCfg<16>::NS * UmmaCfg<16>::NSUB); }
 
 namespace {
-template <typename T, int BITS, bool STATS = false, bool MULTI = false, bool ZOUT = false>
+template <typename T, int BITS, bool STATS = false, bool MULTI = false, bool ZOUT = false, bool SSTATS = false>
 cudaError_t launch_umma_kp(int kpad, const SweepParams& p, const CUtensorMap* tmaps, int* error, int grid, cudaStream_t st) {
+  static_assert(UmmaCfg<16>::EPI_WARPS <= kStatSlots && UmmaCfg<32>::EPI_WARPS <= kStatSlots && UmmaCfg<64>::EPI_WARPS <= kStatSlots,
+                "one bookkeeping slot per epilogue warp");
 #define ZGR_LAUNCH_UMMA(KPV)                                                                                       \
   {                                                                                                                \
-    auto k = sweep_umma_kernel<T, BITS, KPV, STATS, MULTI, ZOUT>;                                                         \
+    auto k = sweep_umma_kernel<T, BITS, KPV, STATS, MULTI, ZOUT, SSTATS>;                                                 \
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<KPV>::SMEM_BYTES); \
     if (e != cudaSuccess) return e;                                                                                \
     k<<<grid, UmmaCfg<KPV>::THREADS, UmmaCfg<KPV>::SMEM_BYTES, st>>>(p, tmaps, error);                                      \
@@ -735,6 +777,10 @@ cudaError_t launch_umma_typed(const KernelChoice& kc, const SweepParams& p, cons
   if (p.n_terms > 1) {
     return kc.bits == 32 ? launch_umma_kp<T, 32, false, true>(kc.kpad, p, tmaps, error, grid, st)
                          : launch_umma_kp<T, 16, false, true>(kc.kpad, p, tmaps, error, grid, st);
+  }
+  if (p.item_stats != nullptr) {   // the sweep also accumulates the norm bookkeeping
+    return kc.bits == 32 ? launch_umma_kp<T, 32, false, false, false, true>(kc.kpad, p, tmaps, error, grid, st)
+                         : launch_umma_kp<T, 16, false, false, false, true>(kc.kpad, p, tmaps, error, grid, st);
   }
   return kc.bits == 32 ? launch_umma_kp<T, 32>(kc.kpad, p, tmaps, error, grid, st) : launch_umma_kp<T, 16>(kc.kpad, p, tmaps, error, grid, st);
 }

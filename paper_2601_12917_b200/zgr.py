@@ -28,7 +28,8 @@ class ZgrTensor(ctypes.Structure):
 
 
 class ZgrConfig(ctypes.Structure):
-    _fields_ = [("alpha", ctypes.c_double), ("eps", ctypes.c_double), ("scale_mode", ctypes.c_int32), ("bits_per_normal", ctypes.c_int32)]
+    _fields_ = [("alpha", ctypes.c_double), ("eps", ctypes.c_double), ("scale_mode", ctypes.c_int32), ("bits_per_normal", ctypes.c_int32),
+                ("stats", ctypes.c_int32)]
 
 
 class ZgrCoeffDelivery(ctypes.Structure):
@@ -80,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.zgr_adapt_alpha.restype = ctypes.c_int
         L.zgr_build_subspace.argtypes = [vp, i32, vp, i32, vp]
         L.zgr_build_subspace.restype = ctypes.c_int
+        L.zgr_enable_stats.argtypes = [vp, i32]
+        L.zgr_enable_stats.restype = ctypes.c_int
         L.zgr_set_coeffs_dtc_rows.argtypes = [vp, i32, vp, vp, vp, i32, i32]
         L.zgr_set_coeffs_dtc_rows.restype = ctypes.c_int
         L.zgr_perturb_layers.argtypes = [vp, u64, dbl, i32, ctypes.POINTER(i32), i32, ctypes.POINTER(ZgrCoeffDelivery), vp, vp]
@@ -139,7 +142,7 @@ class Zgr:
     """
 
     def __init__(self, weights: Sequence, subspaces: Sequence, alpha: float, eps: float, scale_mode: int = SCALE_UNIT,
-                 bits_per_normal: int = 32):
+                 bits_per_normal: int = 32, stats: bool = False):
         assert len(weights) == len(subspaces)
         self._keep: List = [list(weights), list(subspaces)]
         n = len(weights)
@@ -155,7 +158,7 @@ class Zgr:
                     raise ValueError(f"tensor {l}: subspace must be a contiguous CUDA tensor of shape (rows, rank)")
                 rank, uptr = int(U.shape[1]), U.data_ptr()
             arr[l] = ZgrTensor(w.data_ptr(), rows, cols, _dtype_code(w), rank, uptr)
-        cfg = ZgrConfig(alpha, eps, scale_mode, bits_per_normal)
+        cfg = ZgrConfig(alpha, eps, scale_mode, bits_per_normal, 1 if stats else 0)
         self._h = ctypes.c_void_p()
         _check(lib().zgr_init(ctypes.byref(self._h), arr, n, ctypes.byref(cfg)), "zgr_init")
         self.n = n
@@ -276,6 +279,10 @@ class Zgr:
         _check(lib().zgr_profile_read(self._h, arr, 64, ctypes.byref(n)), "zgr_profile_read")
         return [{"path": PATH_NAMES.get(e.path, str(e.path)), "dtype": e.dtype, "kpad": e.kpad, "launches": e.launches,
                  "elements": e.elements, "ms_total": e.ms_total} for e in arr[: n.value]]
+
+    def enable_stats(self, on: bool) -> None:
+        """Keep the norm bookkeeping inside the first perturbation of every seed (zgr_enable_stats)."""
+        _check(lib().zgr_enable_stats(self._h, 1 if on else 0), "zgr_enable_stats")
 
     # -- bookkeeping and test hooks -------------------------------------------------------------
     def get_stats(self, seed: int, stream=None):

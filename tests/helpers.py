@@ -95,7 +95,7 @@ class Pair:
     """The same small model on both sides: device tensors for the library, storage arrays for the oracle."""
 
     def __init__(self, shapes, ranks, dtype: str, alpha=0.5, eps=1e-3, scale_mode=zgr.SCALE_UNIT, bits=32, seed=0, device="cuda",
-                 dtc=None, misalign=False):
+                 dtc=None, misalign=False, stats=False):
         self.dtype, self.device, self.bits = dtype, device, bits
         self.shapes, self.ranks = list(shapes), list(ranks)
         self.theta, self.U, self.q, self.scale, self.zero = [], [], [], [], []
@@ -111,7 +111,7 @@ class Pair:
                 self.theta.append(from_double(w, dtype, (m, n) if m > 1 else (n,), device))
             self.U.append(torch.from_numpy(synth.subspace(m, r, seed * 1000 + l)).to(device) if r > 0 else None)
             self.q.append(None); self.scale.append(None); self.zero.append(None)
-        self.lib = zgr.Zgr(self.theta, self.U, alpha, eps, scale_mode, bits)
+        self.lib = zgr.Zgr(self.theta, self.U, alpha, eps, scale_mode, bits, stats=stats)
         self.alpha, self.eps, self.scale_mode = alpha, eps, scale_mode
         self.d = sum(m * n for m, n in shapes)
         self.K = sum(r * n for (m, n), r in zip(shapes, ranks))

@@ -309,6 +309,47 @@ def test_norm_bookkeeping(bits):
     assert p.lib.state()[0] is False
 
 
+@pytest.mark.parametrize("dtype,bits", [("bf16", 16), ("bf16", 32), ("f16", 16), ("f32", 32)])
+def test_norm_bookkeeping_inside_the_sweep(dtype, bits):
+    """zgr_config.stats: the first perturbation under a seed accumulates the three norms inside its sweep
+    (every kernel family; ragged strips and row blocks), zgr_get_stats then only adds the partial sums up.
+    The sweep itself must still match the oracle, the norms must match oracle.stats_tensor, repeated calls
+    must give identical bits, and the pass of its own (bookkeeping off) must agree."""
+    shapes, ranks = [(64, 256), (1, 100), (40, 72), (48, 128), (300, 392), (130, 1032), (45, 100), (1, 7)], [8, 0, 3, 16, 32, 64, 20, 0]
+    p = Pair(shapes, ranks, dtype, bits=bits, alpha=0.4, stats=True, seed=13)
+    seed, eps = 17, 1e-3
+    launches = p.lib.launch_count()
+    reports = p.call_and_check(seed, eps, lambda: p.lib.perturb(seed, eps), "perturb(+eps) with bookkeeping")
+    assert all(rep["moved"] > 0.3 for rep in reports)
+    swept = p.lib.launch_count() - launches
+    got = p.lib.get_stats(seed)
+    assert p.lib.launch_count() - launches == swept + 1          # one small finishing launch, no pass over the tensors
+    for l in range(len(shapes)):
+        exp = oracle.stats_tensor(p.oracle_tensor(l), seed, l, bits, p.a, p.b)
+        np.testing.assert_allclose(got[l], exp, rtol=2e-5, atol=1e-12)
+    assert np.array_equal(got, p.lib.get_stats(seed))             # fixed summation order
+    # the rest of the step runs without bookkeeping (the seed is active) and still matches the oracle
+    p.call_and_check(seed, -2 * eps, lambda: p.lib.perturb(seed, -2 * eps), "perturb(-2eps)")
+    p.call_and_check(seed, eps, lambda: p.lib.restore_update(seed, 2.0, 2.0, 0.0), "restore")
+    assert np.array_equal(got, p.lib.get_stats(seed))             # still held: nothing that the norms depend on has changed
+    # another seed asked for: a pass of its own; and the same seed through that pass agrees with the sweep's figures
+    other = p.lib.get_stats(seed + 1)
+    exp = oracle.stats_tensor(p.oracle_tensor(4), seed + 1, 4, bits, p.a, p.b)
+    np.testing.assert_allclose(other[4], exp, rtol=2e-5)
+    p.lib.enable_stats(False)
+    p.lib.set_alpha(0.4)                                          # same ratio, but the held norms are dropped
+    by_pass = p.lib.get_stats(seed)
+    np.testing.assert_allclose(by_pass, got, rtol=1e-5, atol=1e-12)
+    assert np.array_equal(by_pass, p.lib.get_stats(seed))
+    # a change of alpha drops the held norms
+    p.lib.enable_stats(True)
+    p.lib.perturb(seed + 2, eps); p.lib.restore_update(seed + 2, 2.0, 2.0, 0.0)
+    p.lib.set_alpha(0.7)
+    a2, b2 = oracle.mix_scalars(0.7, p.d, p.K, p.scale_mode)
+    st = p.lib.get_stats(seed + 2)
+    np.testing.assert_allclose(st[4], oracle.stats_tensor(p.oracle_tensor(4), seed + 2, 4, bits, a2, b2), rtol=2e-5)
+
+
 @pytest.mark.parametrize("dtype,rows,cols,rank", [("f16", 16384, 2048, 16), ("bf16", 8192, 4096, 32), ("bf16", 6144, 1536, 64)])
 def test_many_work_items_per_block(dtype, rows, cols, rank):
     """Tensors cut into ~1000 small work items, several per persistent block: the hand-over between items

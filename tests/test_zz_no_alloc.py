@@ -1,11 +1,12 @@
-"""The allocation-free norms entry point (zgr_tensor_norms_noalloc) against zgr_get_stats.
+"""The allocation-free norms entry point (zgr_tensor_norms_noalloc) against the oracle and against zgr_get_stats.
 
 Some users of the library cannot let it allocate device memory while they run -- an allocation
 forces a device-wide synchronisation that stalls their other streams, or their framework has
 already taken all free device memory for its own pool.  For them the library keeps the scratch of
 this one entry point in a fixed array of its own image.  The test calls it through the C ABI twice in
 a row (the array keeps the previous call's contents, so the second call must not be disturbed by
-the first) and compares with the allocating entry point, within the tolerance of the other norm tests.
+the first) and compares with the oracle's norms and with the allocating entry point, within the tolerance
+of the other norm tests.
 
 Collected last on purpose: a run that stops at the first failure has then already run everything else.
 """
@@ -15,6 +16,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2601_12917_b200 import zgr
 
 from helpers import Pair
@@ -33,6 +35,8 @@ def test_noalloc_norms_match_get_stats_twice_in_a_row():
             torch.cuda.synchronize()
             got = out.cpu().numpy()
             np.testing.assert_allclose(got, ref[l], rtol=2e-5, atol=1e-12)
+            # and against the oracle itself, so that a mistake shared by the two device routes cannot pass
+            np.testing.assert_allclose(got, oracle.stats_tensor(p.oracle_tensor(l), seed, l, 32, p.a, p.b), rtol=2e-5, atol=1e-12)
             # fixed summation order: a repeat gives the same bits
             out2 = torch.empty_like(out)
             p.lib.tensor_norms_noalloc(seed, l, out2)
