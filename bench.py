@@ -9,8 +9,9 @@ perturb(+eps), perturb(-2 eps), restore_update(lr/Q) -- 3Q in-place sweeps over 
 `value` = model parameters stepped per second (parameters x steps / time, all ranks), measured with
 CUDA events with weights, subspaces and work tables resident in HBM.  `e2e` repeats the measurement
 with the per-step inputs coming from the host through the C ABI: every guided tensor's subspace is
-copied from pinned host memory (zgr_update_subspaces), the step runs with the norm bookkeeping kept by its
-first sweep, and the per-tensor norms are read back to the host (zgr_get_stats).  The weights themselves stay in HBM in both: keeping the model on
+copied from pinned host memory, layer by layer on a copy stream while the step's first sweep works through the
+earlier layers (zgr_perturb_layers), that sweep also keeps the norm bookkeeping, and the per-tensor norms are
+read back to the host (zgr_get_stats).  The weights themselves stay in HBM in both: keeping the model on
 the device and never materialising z is the point of the method.
 
 The path does not shard (one GPU holds the model; the only cross-rank quantities would be two loss
@@ -450,9 +451,30 @@ def main():
         d2h = 3 * 8 * len(dm.theta)
         n_e2e = max(1, min(args.steps, 3))
 
+        ends = layer_table(wl)
+        copy_stream = torch.cuda.Stream()
+        deliveries = [(l, None, None, None, host_U[l]) for l in guided]
+
         def e2e_step(t):
-            z.update_subspaces(guided, [host_U[l] for l in guided])
-            run_step(z, wl, t, args.schedule, keep_norms=True)
+            # The step's first sweep runs layer by layer: the subspaces of a layer arrive from pinned host memory
+            # on the copy stream while earlier layers are swept, and that sweep also keeps the norm bookkeeping.
+            if args.schedule == "sequential":
+                seed0 = wl.seed(t, 0)
+                lp, lm = wl.losses(t, 0)
+                z.enable_stats(True)
+                z.perturb_layers(seed0, wl.eps, ends, deliveries, copy_stream=copy_stream)
+                z.enable_stats(False)
+                z.perturb(seed0, -2.0 * wl.eps)
+                z.restore_update(seed0, lp, lm, wl.lr / wl.queries)
+                for q in range(1, wl.queries):
+                    seed = wl.seed(t, q)
+                    lp, lm = wl.losses(t, q)
+                    z.perturb(seed, wl.eps)
+                    z.perturb(seed, -2.0 * wl.eps)
+                    z.restore_update(seed, lp, lm, wl.lr / wl.queries)
+            else:
+                z.update_subspaces(guided, [host_U[l] for l in guided])
+                run_step(z, wl, t, args.schedule, keep_norms=True)
             return z.get_stats(wl.seed(t, 0))      # the norms kept by the step's first sweep: one small launch and a 7 KB read
 
         e2e_step(10_000)
@@ -464,7 +486,7 @@ def main():
         barrier()
         ms_e, units_e = reduce_over_ranks(ev0.elapsed_time(ev1), float(wl.params) * n_e2e, dist if world > 1 else None)
         e2e = {"value": units_e / (ms_e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
-               "ms_per_step": ms_e / n_e2e, "what": "subspaces H2D from pinned memory + step + per-tensor norms D2H, through the C ABI"}
+               "ms_per_step": ms_e / n_e2e, "what": "subspaces H2D from pinned memory (layer by layer on a copy stream, under the step's first sweep) + step + per-tensor norms D2H, through the C ABI"}
 
     # ---- the other configurations, briefly (single process only; the headline above is unaffected) ----
     others = overlap = None

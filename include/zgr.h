@@ -170,26 +170,32 @@ int zgr_set_coeffs_dtc(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const floa
  * 1 <= n_rows <= rank; n_rows = rank is zgr_set_coeffs_dtc.  Errors as there, plus ZGR_EINVAL for n_rows out of range. */
 int zgr_set_coeffs_dtc_rows(zgr_ctx* ctx, int32_t tensor, const int8_t* q, const float* scale, const float* zero, int32_t bits, int32_t n_rows);
 
-/* zgr_perturb, layer by layer, with the compressed coefficients arriving from the host while earlier layers
- * are swept (Sec. 3.3, the layer-wise sample -> transmit -> apply pipeline; Sec. 3.4, the transmission of a
- * layer is to fit under the compute of another).  layer_end: HOST array of n_layers strictly increasing
+/* zgr_perturb, layer by layer, with the guided payload of each layer arriving from the host while earlier
+ * layers are swept (Sec. 3.3, the layer-wise sample -> transmit -> apply pipeline; Sec. 3.4, the transmission
+ * of a layer is to fit under the compute of another).  layer_end: HOST array of n_layers strictly increasing
  * tensor indices, layer L being the tensors [layer_end[L-1], layer_end[L]) and layer_end[n_layers-1] the number
- * of tensors.  deliveries: HOST array; entry i names a tensor whose compressed coefficients were set with
- * zgr_set_coeffs_dtc(_rows) and gives HOST sources (pinned memory, or the copies do not overlap anything) of
- * the same sizes and layout, which are copied into those device buffers on `copy_stream`.  All copies are
- * enqueued at once, in layer order, behind the work already on `stream`; the sweep of a layer on `stream`
- * waits for that layer's copies only, so later layers travel while earlier ones are swept.  n_deliveries = 0
- * gives the same sweep as zgr_perturb, issued as one launch per kernel family and layer.
+ * of tensors.  deliveries: HOST array; entry i names a tensor and gives HOST sources (pinned memory, or the
+ * copies do not overlap anything) for its compressed coefficients (q, scale, zero: the tensor's coefficients
+ * must have been set with zgr_set_coeffs_dtc(_rows); same sizes and layout, copied into those device buffers)
+ * and/or for its subspace (U: rows x rank fp32, copied into the subspace buffer given to zgr_init; the
+ * tensor-core operand copies are rebuilt before the layer is swept).  All copies are enqueued at once on
+ * `copy_stream`, in layer order, behind the work already on `stream`; the sweep of a layer waits for that
+ * layer's copies only, so later layers travel while earlier ones are swept.  Consecutive layers are swept on two
+ * streams in turn (`stream` and one of the library's), which lets a layer start on the SMs that the previous
+ * one has already left; `stream` waits for all of it at the end.  n_deliveries = 0 gives the same sweep as
+ * zgr_perturb, issued as one launch per kernel family and layer.
  * The result is identical to copying everything first and calling zgr_perturb.
- * ZGR_EINVAL: scale not finite, bad layer table, a delivery naming a bad or repeated tensor, a tensor without
- * compressed coefficients, or a zero point given for a tensor registered without one (or the reverse).
- * ZGR_ESTATE: as zgr_perturb; with deliveries, also if any seed is active (coefficients may not change between
+ * ZGR_EINVAL: scale not finite, bad layer table, a delivery naming a bad or repeated tensor or carrying
+ * nothing, coefficients for a tensor without compressed coefficients, a zero point given for a tensor
+ * registered without one (or the reverse), a subspace for a tensor without one.
+ * ZGR_ESTATE: as zgr_perturb; with deliveries, also if any seed is active (the payload may not change between
  * a perturbation and its restore). */
 typedef struct {
   int32_t tensor;
-  const void* q;       /* HOST: codes of the delivered rows */
-  const float* scale;  /* HOST: one per delivered row */
+  const void* q;       /* HOST: codes of the delivered rows, or NULL if only a subspace is delivered */
+  const float* scale;  /* HOST: one per delivered row (NULL iff q is NULL) */
   const float* zero;   /* HOST: one per delivered row, or NULL if the tensor was registered without zero points */
+  const float* U;      /* HOST: rows x rank fp32 subspace, or NULL */
 } zgr_coeff_delivery;
 int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_layers, const int32_t* layer_end, int32_t n_deliveries,
                        const zgr_coeff_delivery* deliveries, void* stream, void* copy_stream);

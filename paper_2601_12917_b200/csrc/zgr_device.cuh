@@ -90,12 +90,35 @@ __device__ __forceinline__ void sincos_quarter_turns(float y, float& sn, float& 
   cs = __int_as_float(__float_as_int(c0) ^ (((q + 1) & 2) << 30));
 }
 
+// -2 ln(u1) for the accurate transform, written for the argument that occurs here: u1 is a multiple of
+// 2^-(nb+1) in (0, 1), so v = 1 - u1 is exact in fp32.
+//   v <= 1/16:  -2 ln(1 - v) = 2 v (1 + v/2 + v^2/3 + ... + v^6/7), truncation below 3e-11, a few fp32 ulp in all.
+//               This is the range where the hardware log2 fails the tolerance: its absolute error of 2^-22 is
+//               a relative error of 1/|log2 u1| 2^-22, unbounded as u1 -> 1, and the square root passes half of it on.
+//   otherwise:  -2 ln 2 * lg2.approx(u1): relative error at most 2.6e-6 (at u1 = 15/16), 2^-22 below 1/2,
+//               i.e. at most 5e-7 absolute on the radius.
+// Both are computed and one is selected (no divergence).  The square root that follows is the hardware one
+// (relative error 2^-23).  Replaces logf and sqrtf, which cost about three times as many instructions.
+__device__ __forceinline__ float neg2_log(float u1) {
+  const float v = 1.0f - u1;                                   // exact
+  float q = fmaf(v, 0.2857142857f, 0.3333333333f);             // 2/7, 2/6
+  q = fmaf(q, v, 0.4f);                                        // 2/5
+  q = fmaf(q, v, 0.5f);                                        // 2/4
+  q = fmaf(q, v, 0.6666666667f);                               // 2/3
+  q = fmaf(q, v, 1.0f);                                        // 2/2
+  q = fmaf(q, v, 2.0f);                                        // 2/1
+  const float near_one = q * v;
+  const float general = -1.3862943611f * lg2_approx(u1);       // -2 ln 2
+  return v <= 0.0625f ? near_one : general;
+}
+
 // m1, m2: the two uniform fields in mantissa position (bits 0..22) under the exponent of 1.0f (field23 / field16a / field16b).
 //
 // PRECISE = false (16-bit weights): hardware log2 / sqrt / sin / cos approximations; absolute error of
 // a unit normal about 4e-6, far below one ulp of the storage type times any step coefficient.
-// PRECISE = true (fp32 weights, tolerance 1e-6 max|theta|): logf, correctly rounded sqrtf and
-// sincos_quarter_turns on the exactly representable angle 4 u2 (in quarter turns), a few fp32 ulp in total.
+// PRECISE = true (fp32 weights, tolerance 1e-6 max|theta|): neg2_log, the hardware square root (2^-23) and
+// sincos_quarter_turns on the exactly representable angle 4 u2 (in quarter turns): below 1e-6 absolute on a
+// unit normal.
 // The fast form cannot serve fp32: besides the sin/cos error, the hardware log2 has an absolute
 // error near 2^-22 for u1 close to 1, which the square root amplifies for the smallest radii.
 template <bool PRECISE>
@@ -105,7 +128,7 @@ __device__ __forceinline__ void box_muller(uint32_t m1, uint32_t m2, const Norma
   if (PRECISE) {
     float sn, cs;
     sincos_quarter_turns(fmaf(4.0f, t2, 4.0f * ns.u1_off), sn, cs);   // 4 u2 in (0, 4), exact
-    const float rho = ns.s * sqrtf(-2.0f * logf(u1));
+    const float rho = ns.s * sqrt_approx(neg2_log(u1));
     n0 = rho * cs;
     n1 = rho * sn;
   } else {

@@ -74,7 +74,8 @@ struct zgr_ctx {
   CUtensorMap* d_tmaps = nullptr;     // three per tensor (theta, U hi, U lo); tcgen05 path only
   std::vector<CUtensorMap> tmaps;     // host mirror
   int* d_err = nullptr;               // set by a kernel whose bounded wait gave up
-  std::vector<cudaEvent_t> layer_events;  // zgr_perturb_layers: one per layer plus one, created on first use
+  std::vector<cudaEvent_t> layer_events;  // zgr_perturb_layers: one per layer plus two, created on first use
+  cudaStream_t aux_stream = nullptr;      // zgr_perturb_layers: odd layers run here, so that one layer's tail overlaps the next one's start
   void* d_qr = nullptr;               // scratch of zgr_build_subspace (grown on demand)
   size_t qr_bytes = 0;
 };
@@ -335,6 +336,28 @@ int flush_descs(zgr_ctx* ctx, cudaStream_t st) {
 }
 
 bool is_finite(double x) { return std::isfinite(x); }
+
+// Rebuild the library's operand copies of U for one tensor from the subspace buffer (enqueued on st).
+int refresh_operands(zgr_ctx* ctx, int32_t tensor, cudaStream_t st) {
+  TensorDesc& td = ctx->descs[static_cast<size_t>(tensor)];
+  int rc = ZGR_OK;
+  if (td.Ufrag != nullptr) {
+    if (td.umma) {
+      // the sweeps of this tensor read the row-major copy below; the fragment-order copy is only needed by
+      // zgr_debug_z and is rebuilt there on demand
+      ctx->frag_stale[static_cast<size_t>(tensor)] = 1;
+    } else {
+      rc = check(ctx, launch_split_subspace(td.U, td.rows, td.rank, td.kpad, const_cast<uint4*>(td.Ufrag), st));
+      if (rc == ZGR_OK) ctx->launches++;
+    }
+  }
+  if (rc == ZGR_OK && td.umma) {
+    const int64_t rows_pad = ((td.rows + 127) / 128) * 128;
+    rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.ushift, td.Uhi, td.Ulo, st));
+    if (rc == ZGR_OK) ctx->launches++;
+  }
+  return rc;
+}
 
 // Bookkeeping slots of a plan: kStatSlots x 3 doubles per work item, zeroed once (slots that no warp owns stay
 // zero; the others are rewritten by every launch that keeps the bookkeeping).
@@ -744,10 +767,12 @@ int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_laye
   std::vector<char> seen(static_cast<size_t>(n), 0);
   for (int32_t i = 0; i < n_deliveries; ++i) {
     const zgr_coeff_delivery& d = deliveries[i];
-    if (d.tensor < 0 || d.tensor >= n || seen[static_cast<size_t>(d.tensor)] || !d.q || !d.scale) return ZGR_EINVAL;
+    if (d.tensor < 0 || d.tensor >= n || seen[static_cast<size_t>(d.tensor)] || (!d.q && !d.U)) return ZGR_EINVAL;
     seen[static_cast<size_t>(d.tensor)] = 1;
     const TensorDesc& td = ctx->descs[static_cast<size_t>(d.tensor)];
-    if (td.q == nullptr || (d.zero != nullptr) != (td.qzero != nullptr)) return ZGR_EINVAL;
+    if (d.q && (!d.scale || td.q == nullptr || (d.zero != nullptr) != (td.qzero != nullptr))) return ZGR_EINVAL;
+    if (!d.q && (d.scale || d.zero)) return ZGR_EINVAL;
+    if (d.U && td.rank == 0) return ZGR_EINVAL;
     const int32_t L = static_cast<int32_t>(std::upper_bound(layer_end, layer_end + n_layers, d.tensor) - layer_end);
     by_layer[static_cast<size_t>(L)].push_back(i);
   }
@@ -757,7 +782,11 @@ int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_laye
   cudaStream_t st = static_cast<cudaStream_t>(stream), cs = static_cast<cudaStream_t>(copy_stream);
   int rc = flush_descs(ctx, st);
   if (rc != ZGR_OK) return rc;
-  while (ctx->layer_events.size() < static_cast<size_t>(n_layers) + 1) {
+  if (!ctx->aux_stream) {
+    rc = check(ctx, cudaStreamCreateWithFlags(&ctx->aux_stream, cudaStreamNonBlocking));
+    if (rc != ZGR_OK) return rc;
+  }
+  while (ctx->layer_events.size() < static_cast<size_t>(n_layers) + 2) {
     cudaEvent_t e = nullptr;
     rc = check(ctx, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     if (rc != ZGR_OK) return rc;
@@ -776,11 +805,15 @@ int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_laye
         const zgr_coeff_delivery& d = deliveries[i];
         const TensorDesc& td = ctx->descs[static_cast<size_t>(d.tensor)];
         const size_t row_bytes = td.qbits == 4 ? static_cast<size_t>((td.cols + 1) / 2) : static_cast<size_t>(td.cols);
-        rc = check(ctx, cudaMemcpyAsync(const_cast<int8_t*>(td.q), d.q, row_bytes * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
-        if (rc == ZGR_OK)
-          rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.qscale), d.scale, sizeof(float) * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
-        if (rc == ZGR_OK && d.zero)
-          rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.qzero), d.zero, sizeof(float) * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
+        if (d.q) {
+          rc = check(ctx, cudaMemcpyAsync(const_cast<int8_t*>(td.q), d.q, row_bytes * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
+          if (rc == ZGR_OK)
+            rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.qscale), d.scale, sizeof(float) * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
+          if (rc == ZGR_OK && d.zero)
+            rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.qzero), d.zero, sizeof(float) * static_cast<size_t>(td.qrows), cudaMemcpyHostToDevice, cs));
+        }
+        if (rc == ZGR_OK && d.U)
+          rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.U), d.U, sizeof(float) * static_cast<size_t>(td.rows) * td.rank, cudaMemcpyHostToDevice, cs));
         if (rc != ZGR_OK) return rc;
       }
       rc = check(ctx, cudaEventRecord(ctx->layer_events[static_cast<size_t>(L)], cs));
@@ -793,13 +826,32 @@ int zgr_perturb_layers(zgr_ctx* ctx, uint64_t seed, double scale, int32_t n_laye
     if (rc != ZGR_OK) return rc;
   }
   ctx->held_valid = false;     // (a delivery changes the coefficients that earlier norms were taken with)
+  // Layers touch disjoint tensors, so consecutive layers need no ordering between them: even layers run on the
+  // caller's stream, odd ones on a stream of the library's, and the blocks of one layer's kernels start on the
+  // SMs that the previous layer's last blocks have not reached any more.  The library's stream starts behind the
+  // work already on the caller's stream, and the caller's stream ends by waiting for it.
+  cudaEvent_t ev_begin = ctx->layer_events[static_cast<size_t>(n_layers) + 1];
+  rc = check(ctx, cudaEventRecord(ev_begin, st));
+  if (rc == ZGR_OK) rc = check(ctx, cudaStreamWaitEvent(ctx->aux_stream, ev_begin, 0));
+  if (rc != ZGR_OK) return rc;
   for (int32_t L = 0; L < n_layers; ++L) {
+    cudaStream_t ls = (L & 1) ? ctx->aux_stream : st;
     if (n_deliveries > 0 && !by_layer[static_cast<size_t>(L)].empty()) {
-      rc = check(ctx, cudaStreamWaitEvent(st, ctx->layer_events[static_cast<size_t>(L)], 0));
+      rc = check(ctx, cudaStreamWaitEvent(ls, ctx->layer_events[static_cast<size_t>(L)], 0));
       if (rc != ZGR_OK) return rc;
+      for (int32_t i : by_layer[static_cast<size_t>(L)])
+        if (deliveries[i].U) {
+          rc = refresh_operands(ctx, deliveries[i].tensor, ls);   // the delivered subspace, split for the tensor cores
+          if (rc != ZGR_OK) return rc;
+        }
     }
-    rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, st, L ? layer_end[L - 1] : 0, layer_end[L], keep);
+    rc = sweep(ctx, ctx->groups, ctx->d_descs, 1, &seed, &scale, ls, L ? layer_end[L - 1] : 0, layer_end[L], keep);
     if (rc != ZGR_OK) return rc;   // (a failure here leaves the earlier layers swept: the context is sticky-failed by check())
+  }
+  if (n_layers > 1) {
+    rc = check(ctx, cudaEventRecord(ev_begin, ctx->aux_stream));
+    if (rc == ZGR_OK) rc = check(ctx, cudaStreamWaitEvent(st, ev_begin, 0));
+    if (rc != ZGR_OK) return rc;
   }
   if (keep) {
     ctx->held_valid = true;
@@ -1053,22 +1105,7 @@ int zgr_update_subspace(zgr_ctx* ctx, int32_t tensor, const float* U_src, int32_
     rc = check(ctx, cudaMemcpyAsync(const_cast<float*>(td.U), U_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, st));
     if (rc != ZGR_OK) return rc;
   }
-  if (td.Ufrag != nullptr) {
-    if (td.umma) {
-      // the sweeps of this tensor read the row-major copy below; the fragment-order copy is only needed by
-      // zgr_debug_z and is rebuilt there on demand
-      ctx->frag_stale[static_cast<size_t>(tensor)] = 1;
-    } else {
-      rc = check(ctx, launch_split_subspace(td.U, td.rows, td.rank, td.kpad, const_cast<uint4*>(td.Ufrag), st));
-      if (rc == ZGR_OK) ctx->launches++;
-    }
-  }
-  if (rc == ZGR_OK && td.umma) {
-    const int64_t rows_pad = ((td.rows + 127) / 128) * 128;
-    rc = check(ctx, launch_split_subspace_rowmajor(td.U, td.rows, td.rank, td.kpad, rows_pad, td.ushift, td.Uhi, td.Ulo, st));
-    if (rc == ZGR_OK) ctx->launches++;
-  }
-  return rc;
+  return refresh_operands(ctx, tensor, st);
 }
 
 int zgr_build_subspace(zgr_ctx* ctx, int32_t tensor, const float* grads, int32_t src_is_host, void* stream) {
@@ -1282,6 +1319,7 @@ void zgr_destroy(zgr_ctx* ctx) {
         cudaEventDestroy(ev.second);
       }
   for (cudaEvent_t e : ctx->layer_events) cudaEventDestroy(e);
+  if (ctx->aux_stream) cudaStreamDestroy(ctx->aux_stream);
   for (void* p : ctx->owned) cudaFree(p);
   delete ctx;
 }

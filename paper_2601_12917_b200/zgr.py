@@ -33,7 +33,7 @@ class ZgrConfig(ctypes.Structure):
 
 
 class ZgrCoeffDelivery(ctypes.Structure):
-    _fields_ = [("tensor", ctypes.c_int32), ("q", ctypes.c_void_p), ("scale", ctypes.c_void_p), ("zero", ctypes.c_void_p)]
+    _fields_ = [("tensor", ctypes.c_int32), ("q", ctypes.c_void_p), ("scale", ctypes.c_void_p), ("zero", ctypes.c_void_p), ("U", ctypes.c_void_p)]
 
 
 class ZgrKernelTime(ctypes.Structure):
@@ -226,12 +226,17 @@ class Zgr:
     def perturb_layers(self, seed: int, scale: float, layer_end: Sequence[int], deliveries=(), stream=None, copy_stream=None) -> None:
         """Layer-wise perturbation with the compressed coefficients of each layer arriving from the host on
         `copy_stream` while earlier layers are swept (zgr_perturb_layers).  deliveries: tuples
-        (tensor, q_host, scale_host, zero_host or None) of host tensors (pinned for overlap)."""
+        (tensor, q_host, scale_host, zero_host or None[, U_host or None]) of host tensors (pinned for overlap);
+        q_host / scale_host may be None when only a subspace travels."""
         nl, nd = len(layer_end), len(deliveries)
         arr = (ZgrCoeffDelivery * max(nd, 1))()
-        for i, (l, q, sc, ze) in enumerate(deliveries):
-            assert not q.is_cuda and not sc.is_cuda and q.is_contiguous() and sc.is_contiguous()
-            arr[i] = ZgrCoeffDelivery(l, q.data_ptr(), sc.data_ptr(), None if ze is None else ze.data_ptr())
+        for i, d in enumerate(deliveries):
+            l, q, sc, ze = d[:4]
+            U = d[4] if len(d) > 4 else None
+            for h in (q, sc, ze, U):
+                assert h is None or (not h.is_cuda and h.is_contiguous())
+            arr[i] = ZgrCoeffDelivery(l, None if q is None else q.data_ptr(), None if sc is None else sc.data_ptr(),
+                                      None if ze is None else ze.data_ptr(), None if U is None else U.data_ptr())
         self._keep.append(list(deliveries))
         if copy_stream is None:
             import torch

@@ -94,6 +94,42 @@ def test_layerwise_delivery_matches_the_oracle_and_the_plain_sweep(omega, bits, 
     assert a.lib.state()[0] is False
 
 
+def test_layerwise_delivery_of_subspaces():
+    """The subspaces themselves can travel the same way: a delivered U is copied into the tensor's subspace
+    buffer and split for the tensor cores before its layer is swept."""
+    a = Pair(SHAPES, RANKS, "bf16", bits=16, seed=3, stats=True)
+    new_U = {l: torch.from_numpy(synth.subspace(SHAPES[l][0], RANKS[l], 900 + l)).pin_memory() for l in range(len(SHAPES)) if RANKS[l]}
+    copy_stream = torch.cuda.Stream()
+    deliveries = [(l, None, None, None, U) for l, U in new_U.items()]
+    seed, eps = 21, 1e-3
+    ots = [a.oracle_tensor(l) for l in range(len(SHAPES))]
+    a.lib.perturb_layers(seed, eps, LAYER_END, deliveries, copy_stream=copy_stream)
+    torch.cuda.synchronize()
+    assert a.lib.device_status() == 0
+    from helpers import check_sweep, to_double
+    for l, t in enumerate(ots):
+        assert RANKS[l] == 0 or torch.equal(a.U[l].cpu(), new_U[l])          # the subspace buffer holds what arrived
+        before = oracle.decode(t.theta, t.dtype)
+        t2 = a.oracle_tensor(l)
+        t2.theta = t.theta
+        oracle.sweep_tensor(t2, seed, l, 16, a.a, a.b, eps)
+        rep = check_sweep(to_double(a.theta[l]), oracle.decode(t2.theta, t2.dtype), before, "bf16", 1.0, f"perturb_layers(U) tensor {l}",
+                          operand=eps * a.sigma_z(l), c_abs=eps)
+        assert rep["moved"] > 0.3
+    # the norms kept by that layer-wise sweep are those of the delivered subspaces
+    st = a.lib.get_stats(seed)
+    for l in range(len(SHAPES)):
+        np.testing.assert_allclose(st[l], oracle.stats_tensor(a.oracle_tensor(l), seed, l, 16, a.a, a.b), rtol=2e-5, atol=1e-12)
+    a.call_and_check(seed, -2 * eps, lambda: a.lib.perturb(seed, -2 * eps), "perturb(-2eps)")
+    a.call_and_check(seed, eps, lambda: a.lib.restore_update(seed, 2.0, 2.0, 0.0), "restore")
+    with pytest.raises(zgr.ZgrError) as e:                      # a subspace for a vector
+        a.lib.perturb_layers(5, eps, LAYER_END, [(1, None, None, None, new_U[0])], copy_stream=copy_stream)
+    assert e.value.code == zgr.EINVAL
+    with pytest.raises(zgr.ZgrError) as e:                      # a delivery that carries nothing
+        a.lib.perturb_layers(5, eps, LAYER_END, [(0, None, None, None, None)], copy_stream=copy_stream)
+    assert e.value.code == zgr.EINVAL
+
+
 def test_layer_table_and_delivery_errors():
     p = Pair(SHAPES[:3], RANKS[:3], "bf16", bits=16)
     q, sc = synth.dtc_payload(32, 392, seed=1)
