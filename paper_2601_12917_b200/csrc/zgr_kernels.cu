@@ -28,6 +28,11 @@ namespace zgr {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 
+// Rows ahead that the CUDA-core kernel prefetches into L2 (0 = off).
+#ifndef ZGR_FMA_PREFETCH
+#define ZGR_FMA_PREFETCH 2
+#endif
+
 // ---------------------------------------------------------------------------------------------
 // isotropic sweep
 // ---------------------------------------------------------------------------------------------
@@ -112,6 +117,14 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_con
     const int64_t row_end = w.row0_or_e0 + w.nrows_or_count;
     double s_iso = 0.0, s_gd = 0.0, s_z = 0.0;   // SSTATS only
     for (int64_t row = w.row0_or_e0 + warp; row < row_end; row += kWarps) {
+#if ZGR_FMA_PREFETCH
+      // this warp's row after next: start it on its way from HBM to L2 now (each lane asks for its own 8 elements);
+      // with four warps per scheduler there is not enough other work to cover a full DRAM round trip otherwise
+      if (active && row + ZGR_FMA_PREFETCH * kWarps < row_end) {
+        const T* nxt = base + (row + ZGR_FMA_PREFETCH * kWarps) * cols + w.col0 + 8 * lane;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(nxt));
+      }
+#endif
       float u[R];
       if (u_vec) {
 #pragma unroll

@@ -61,3 +61,24 @@ def test_sequential_and_deferred_schedules_agree():
     assert passes == [2 * 3 * wl.queries, 2 * (2 * wl.queries + 1)]
     np.testing.assert_allclose(results[1], results[0], rtol=0, atol=1e-14)
     assert np.abs(results[0]).max() > 0
+
+
+def test_layer_table_covers_every_tensor_once():
+    """The layer table that bench.py hands to zgr_perturb_layers: strictly increasing, ends at the number of
+    tensors, one layer for what precedes the blocks, one per Transformer block, one for what follows them."""
+    expected_layers = {"roberta_large": 25, "opt_1p3b": 26, "llama_7b": 34, "llama_13b": 42}
+    for name, n_layers in expected_layers.items():
+        wl = synth.workload(name)
+        ends = bench.layer_table(wl)
+        assert len(ends) == n_layers and ends[-1] == len(wl.tensors)
+        assert all(b > a for a, b in zip([0] + ends[:-1], ends))
+        # a block's tensors share their name prefix, and no prefix is split over two layers
+        start = 0
+        seen = set()
+        for end in ends:
+            prefixes = {t.name.split(".")[0] for t in wl.tensors[start:end]}
+            blocks = {p for p in prefixes if p.startswith("l") and p[1:].isdigit()}
+            assert len(blocks) <= 1 and (not blocks or prefixes == blocks)
+            assert not (prefixes & seen)
+            seen |= prefixes
+            start = end
