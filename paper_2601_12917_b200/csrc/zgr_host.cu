@@ -285,7 +285,6 @@ int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, i
   p.n_terms = n;
   p.unit = make_scale(1.0, ctx->cfg.bits_per_normal);
   p.tensors = d_descs;
-  p.stats = nullptr;
   double cb_total = 0.0;
   for (int q = 0; q < n; ++q) cb_total += std::fabs(c[q] * ctx->b);
   p.kshift = kshift_for(cb_total);

@@ -74,7 +74,6 @@ struct SweepParams {
   const TensorDesc* tensors;
   const WorkItem* items;
   int32_t n_items;
-  double* stats;         // 3 doubles per tensor (stats kernels only)
   float* zout;           // rows x cols fp32 image of the one tensor swept (test hook of the tcgen05 kernel only)
   double* item_stats;    // norm bookkeeping: kStatSlots x 3 doubles per work item of the group (partial sums per warp), or null
   int32_t item_base;     // index of items[0] in the group's full item list (layer-wise launches start in the middle)

@@ -5,12 +5,12 @@
 // HBM can feed the weights, so everything else is taken out of the SM's instruction stream:
 //
 //   * TMA brings a 128-row x NS-column tile of theta (and the matching 128 x KP tiles of U, pre-split
-//     into bf16 hi/lo) into shared memory, and writes the finished tile back; no thread issues a
+//     into fp16 hi/lo) into shared memory, and writes the finished tile back; no thread issues a
 //     global load or store for the weights.
 //   * tcgen05.mma builds   D = theta + c b U G   in tensor memory (fp32):
 //       - "theta" enters through identity products  D[:, 16j:16j+16] = theta[:, 16j:16j+16] * I16
 //         with theta's own 16-bit tile as the A operand, which unpacks it to fp32 exactly, for free;
-//       - U G is formed first as  Ulo Ghi + Uhi Glo + Uhi Ghi  with fp16 split operands (hi + lo carries 22
+//       - U G is formed first, as  Ulo Ghi + Uhi Glo + Uhi Ghi  with fp16 split operands (hi + lo carries 22
 //         significant bits, against 16 for a bf16 split, whose representation error of 4.5e-6 relative was the
 //         whole error of z on this path).  fp16 has a narrow exponent range, so both operands are kept near 1
 //         by powers of two: the library's copy of U holds U 2^j (j from the tensor's row count), the strips hold
@@ -325,7 +325,7 @@ struct TileCoord {
 // that a CTA touches up to 256*NSUB contiguous bytes of every row and loads each U tile once.
 // STATS = true turns the same pipeline into the norm bookkeeping: no weights are loaded or stored,
 // D = b U G only, and the epilogue accumulates sum (a Z)^2, sum (b U G)^2 and sum z^2 per tensor
-// (term[0].iso carries the scale a, term[0].cb = b, p.stats the three doubles per tensor).
+// (term[0].iso carries the scale a, term[0].cb = b; the sums go to the work item's bookkeeping slots).
 // MULTI = true applies several (seed, coefficient) terms in the one pass: the coefficient strips of
 // the terms are summed before the split (U (sum_q c_q b G_q) is one product), the isotropic normals
 // are added term by term in the epilogue.

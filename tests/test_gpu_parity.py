@@ -53,7 +53,7 @@ Z_CASES = [
     ((45, 100), 20, "generic", "generic, high rank"),
 ]
 # absolute tolerance on a unit-variance z: fp32 tensors use the accurate transform and an exact fp32
-# contraction; 16-bit tensors use the hardware approximations and, above rank 8, split-bf16 tensor cores
+# contraction; 16-bit tensors use the hardware approximations and, above rank 8, split 16-bit operands on tensor cores
 Z_TOL = {("f32", "iso"): 2e-6, ("f32", "fma"): 2e-6, ("f32", "mma"): 3e-6, ("f32", "generic"): 3e-6,
          ("bf16", "iso"): 1e-5, ("bf16", "fma"): 1e-5, ("bf16", "mma"): 4e-5, ("bf16", "generic"): 1e-5}
 # ("mma" rows: zgr_debug_z runs the legacy mma.sync kernel for these tensors, whose operands are split into bf16

@@ -3,7 +3,7 @@
 zgr_debug_z runs 16-bit tensors of rank > 8 through the legacy mma.sync kernel (it sweeps an fp32 image,
 which the tcgen05 kernel cannot read), so it says nothing about the kernel that carries the OPT- and
 LLaMA-shaped configurations.  zgr_debug_z_tcgen05 runs that kernel (TMA loads of a zeroed 16-bit image,
-identity products, the three split-bf16 products of U G, tensor-memory reads, generator and Gaussian
+the three split-fp16 products of U G, identity products, tensor-memory reads, generator and Gaussian
 transform in the epilogue) and hands back its fp32 result before the rounding to the storage type.
 
 Bounds (absolute, z of unit variance):
