@@ -40,7 +40,7 @@ UNIT = "params/s"
 NCU_TRAFFIC = {"kernel": "sweep_umma_kernel(k=32)", "workload": "llama_7b", "bytes_per_launch": 26.75e9,
                "sources": ["paper_2601_12917_b200/csrc/zgr_umma.cu", "paper_2601_12917_b200/csrc/zgr_device.cuh",
                            "paper_2601_12917_b200/csrc/zgr_internal.h"],
-               "sha1": "c6528b1bcb3820c52be570c99a09732992cd2bde"}
+               "sha1": "6b5749836414c60e4212f96ea4d0513a440a50e2"}
 
 
 def _code_only(text: str) -> str:

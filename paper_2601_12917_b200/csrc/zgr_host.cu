@@ -28,6 +28,7 @@ struct Group {
   int grid = 0;
   int64_t elements = 0;                                   // weights covered by one launch
   double* d_item_stats = nullptr;                         // kStatSlots x 3 doubles per item (norm bookkeeping), allocated on first use
+  int32_t* d_sched = nullptr;                             // CUDA-core contraction kernel: two item counters (caller's stream, library's second stream)
   std::vector<int32_t> first_item;                        // per tensor l: index of its first item in `items` (size n + 1; items are in tensor order)
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed;  // per-launch events while profiling is on
 };
@@ -218,7 +219,9 @@ void plan(const std::vector<TensorDesc>& descs, const std::vector<int>& which, b
     Group& g = group_for(path, t.dtype, kpad);
     for (int64_t c0 = 0; c0 < t.cols; c0 += strip) {
       const int ncols = static_cast<int>(std::min<int64_t>(strip, t.cols - c0));
-      int64_t nrows = std::max<int64_t>(1, (path == PATH_UMMA ? 2 * target : target) / ncols);
+      // (the CUDA-core contraction kernel hands its items out dynamically and regenerates its coefficient strip per item:
+      //  larger items there; the tcgen05 kernel's items are two tiles wide)
+      int64_t nrows = std::max<int64_t>(1, (path == PATH_UMMA || path == PATH_FMA ? 2 * target : target) / ncols);
       nrows = ((nrows + row_step - 1) / row_step) * row_step;
       // even out the chunks of this strip
       const int64_t n_chunks = (t.rows + nrows - 1) / nrows;
@@ -267,8 +270,15 @@ int upload_groups(zgr_ctx* ctx, std::vector<Group>& groups) {
     if (rc != ZGR_OK) return rc;
     rc = check(ctx, cudaMemcpy(g.d_items, g.items.data(), g.items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
     if (rc != ZGR_OK) return rc;
+    if (g.kc.path == PATH_FMA) {
+      rc = dev_alloc(ctx, &g.d_sched, 2);
+      if (rc != ZGR_OK) return rc;
+      rc = check(ctx, cudaMemset(g.d_sched, 0, 2 * sizeof(int32_t)));
+      if (rc != ZGR_OK) return rc;
+    }
   }
-  return ZGR_OK;
+  // the copies and the zeroing above are not ordered with launches on the caller's (possibly non-blocking) streams
+  return check(ctx, cudaDeviceSynchronize());
 }
 
 // One sweep  theta <- rnd(theta + sum_q c_q z(seed_q))  over the planned groups (n terms, 1 <= n <= kMaxTerms).
@@ -294,6 +304,7 @@ int sweep(zgr_ctx* ctx, std::vector<Group>& groups, const TensorDesc* d_descs, i
     p.n_items = static_cast<int32_t>(g.items.size());
     p.item_stats = keep_stats ? g.d_item_stats : nullptr;
     p.item_base = 0;
+    p.sched = g.d_sched ? g.d_sched + (ctx->aux_stream != nullptr && st == ctx->aux_stream ? 1 : 0) : nullptr;
     int grid = g.grid;
     if (t1 >= 0) {
       const int32_t b0 = g.first_item[static_cast<size_t>(t0)], b1 = g.first_item[static_cast<size_t>(t1)];

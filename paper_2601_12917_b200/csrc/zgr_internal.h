@@ -77,6 +77,7 @@ struct SweepParams {
   float* zout;           // rows x cols fp32 image of the one tensor swept (test hook of the tcgen05 kernel only)
   double* item_stats;    // norm bookkeeping: kStatSlots x 3 doubles per work item of the group (partial sums per warp), or null
   int32_t item_base;     // index of items[0] in the group's full item list (layer-wise launches start in the middle)
+  int32_t* sched;        // CUDA-core contraction kernel: this launch's item counter (zero between launches), see sweep_fma_kernel
   int32_t kshift;        // tcgen05 kernel: the coefficient strips are scaled by a power of two so that sum_q |c_q| b 2^kshift
                          // is near 1 (see the operand precision note in zgr_umma.cu)
 };

@@ -83,15 +83,28 @@ __global__ void __launch_bounds__(kThreads) sweep_iso_kernel(const __grid_consta
 template <typename T, int BITS, bool PRECISE, int R, bool MULTI, bool SSTATS = false>
 __global__ void __launch_bounds__(kThreads, 2) sweep_fma_kernel(const __grid_constant__ SweepParams p) {
   __shared__ float Gs[R][256 + 8];
+  __shared__ int next_item;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int it = blockIdx.x; it < p.n_items; it += gridDim.x) {
+  for (;;) {
+    // Items are handed out in order by a counter in global memory: the models this kernel serves have few items per
+    // CTA (about 18 for a RoBERTa-large-sized set), so a fixed assignment leaves the SMs that drew one item fewer
+    // idle for 3-5 % of the sweep.  Every CTA makes exactly one fetch beyond the end; the last of those puts the
+    // counter back to zero for the next launch (launches that share a counter are ordered by their stream).
+    __syncthreads();  // readers of the previous strip and of next_item are done
+    if (threadIdx.x == 0) {
+      const int t = atomicAdd(p.sched, 1);
+      if (t == p.n_items + static_cast<int>(gridDim.x) - 1) *p.sched = 0;
+      next_item = t;
+    }
+    __syncthreads();
+    const int it = next_item;
+    if (it >= p.n_items) break;
     const WorkItem w = p.items[it];
     const TensorDesc& td = p.tensors[w.tensor];
     T* base = static_cast<T*>(td.data);
     const uint32_t tid = static_cast<uint32_t>(td.id);
     const int r = td.rank;
     const int64_t cols = td.cols;
-    __syncthreads();  // readers of the previous strip are done
     for (int idx = threadIdx.x; idx < R * 32; idx += kThreads) {
       const int k = idx >> 5, o = idx & 31;
       if (8 * o < w.ncols) {
