@@ -156,3 +156,34 @@ def test_layer_table_and_delivery_errors():
     p.lib.perturb_layers(1, -2e-3, [1, 3], copy_stream=cs)
     p.lib.restore_update(1, 2.0, 2.0, 0.0)
     assert p.lib.state()[0] is False
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_layerwise_sweeps_of_low_rank_tensors_on_both_streams(dtype):
+    """Every layer holds tensors of rank <= 8, so consecutive layers run the CUDA-core contraction kernel on the two
+    alternating streams at the same time; that kernel hands its work items out through a counter per stream, which
+    each launch must leave at zero for the next one.  Many layers of different sizes, layer-wise and whole-model
+    sweeps in turn, every call against the oracle and against a context that only ever sweeps the whole model."""
+    shapes, ranks, ends = [], [], []
+    for L in range(9):
+        shapes += [(96 + 40 * L, 264 + 256 * (L % 3)), (1, 72 + 8 * L), (64 + 8 * L, 520)]
+        ranks += [8, 0, 4 if L % 2 else 6]
+        ends.append(len(shapes))
+    a = Pair(shapes, ranks, dtype, bits=16, seed=12)
+    b = Pair(shapes, ranks, dtype, bits=16, seed=12)
+    eps = 1e-3
+    for step, seed in enumerate((5, 6, 7)):
+        a.call_and_check(seed, eps, lambda: a.lib.perturb_layers(seed, eps, ends), f"perturb_layers(+eps) step {step}")
+        b.lib.perturb(seed, eps)
+        if step == 1:
+            a.call_and_check(seed, -2 * eps, lambda: a.lib.perturb(seed, -2 * eps), f"perturb(-2eps) step {step}")
+        else:
+            a.call_and_check(seed, -2 * eps, lambda: a.lib.perturb_layers(seed, -2 * eps, ends), f"perturb_layers(-2eps) step {step}")
+        b.lib.perturb(seed, -2 * eps)
+        c = eps - 1e-4 * oracle.projected_grad(2.3, 1.8, eps)
+        a.call_and_check(seed, c, lambda: a.lib.restore_update(seed, 2.3, 1.8, 1e-4), f"restore_update step {step}")
+        b.lib.restore_update(seed, 2.3, 1.8, 1e-4)
+        torch.cuda.synchronize()
+        for l in range(len(shapes)):
+            assert torch.equal(a.theta[l], b.theta[l]), f"step {step} tensor {l}"
+    assert a.lib.device_status() == 0 and a.lib.state()[0] is False
