@@ -19,7 +19,9 @@
  *
  * Conventions.
  *   - Every `void* stream` is a cudaStream_t (NULL = the legacy default stream).  Sweeps are
- *     enqueued on it and return without synchronising.
+ *     enqueued on it and return without synchronising.  The sweeps of one context must be ordered
+ *     with respect to each other (one stream, or streams that the caller orders): they write the
+ *     same weights and share the library's work-item counters.
  *   - "device" pointers are CUDA device addresses on the current device; the library never
  *     dereferences them on the host and never frees them.  They are borrowed for the life of the
  *     context.
